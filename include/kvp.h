@@ -1,0 +1,209 @@
+/*
+ * kvp.h - C ABI of the composed-cache query-prefill library (KV Packet serving path) for NVIDIA B200.
+ *
+ * The paper's serving step (Section 3.1; Section 3.2 step 4): N document KV caches ("packets"), each
+ * computed offline and wrapped in header/trailer soft-token adapters (Eq. 2), are re-aligned to their
+ * positions in the request by one RoPE rotation per key (Eq. 1), concatenated without recomputation,
+ * and the query tokens then attend causally over everything before them (Fig. 2(d)).
+ *
+ * Conventions
+ *   - every call returns a kvp_status (0 = KVP_OK); nothing throws, aborts or traps the device;
+ *   - all argument checking happens on the host before any kernel is launched;
+ *   - kernels are enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
+ *     stream) and the call returns without synchronising unless stated;
+ *   - "device" pointers are CUDA device addresses on the context's GPU, "host" pointers are ordinary
+ *     host addresses; the library never allocates device memory: the caller lends it a pool and a
+ *     workspace at kvp_create and keeps them alive until kvp_destroy;
+ *   - ids are dense int32 counted from 0 in registration order;
+ *   - element type is the context's dtype (float32 or bfloat16) for every K/V/Q/out buffer.
+ */
+#ifndef KVP_H_
+#define KVP_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define KVP_API __attribute__((visibility("default")))
+#else
+#define KVP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum kvp_status {
+    KVP_OK = 0,
+    KVP_ERR_INVALID = 1,      /* bad argument (null pointer, out-of-range value, bad CSR)          */
+    KVP_ERR_CAPACITY = 2,     /* pool, workspace or a configured maximum would be exceeded         */
+    KVP_ERR_NOT_FOUND = 3,    /* unknown packet / adapter / assembly id                            */
+    KVP_ERR_STATE = 4,        /* call not possible in this state (e.g. host-only context)          */
+    KVP_ERR_UNSUPPORTED = 5,  /* valid request that this build has no kernel for                   */
+    KVP_ERR_CUDA = 6,         /* a CUDA runtime/driver call failed (text in kvp_last_error)        */
+    KVP_ERR_TIMEOUT = 7       /* a bounded device-side wait ran out (see kvp_status_word)          */
+} kvp_status;
+
+enum { KVP_DTYPE_F32 = 0, KVP_DTYPE_BF16 = 1 };
+
+/* kvp_assemble flags */
+enum {
+    KVP_REBASE = 1u,          /* rotate every cached key from its cache-time position to its slot (Eq. 1) */
+    KVP_MATERIALIZE = 2u      /* also copy the whole composed prefix into the workspace cache             */
+};
+
+/* kvp_query_prefill flags */
+enum {
+    KVP_ROPE_QUERY = 1u,      /* q and k_new are raw: rotate them at positions prefix_len[b] + i        */
+    KVP_FORCE_SIMPLE = 2u     /* use the plain fp32 CUDA-core kernel (cross-check path, any dtype)      */
+};
+
+typedef struct kvp_ctx kvp_ctx;
+
+typedef struct kvp_config {
+    int32_t struct_bytes;       /* = sizeof(kvp_config)                                               */
+    int32_t device;             /* CUDA device ordinal; -1 = host-only planning context: registration
+                                   records sizes, kvp_assemble/kvp_export_plan work, nothing can run  */
+    int32_t n_layers;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;         /* must divide n_q_heads; q head h reads kv head h / (Hq/Hkv)         */
+    int32_t head_dim;           /* 64 or 128                                                          */
+    int32_t dtype;              /* KVP_DTYPE_*                                                        */
+    int32_t rope_pairing;       /* 0: pairs (i, i + d/2);  1: pairs (2i, 2i + 1)                      */
+    double rope_theta;          /* theta_i = rope_theta^(-2i/d), i < d/2                              */
+    const double *inv_freq;     /* optional host array [head_dim/2] overriding rope_theta; copied     */
+    double softmax_scale;       /* 0 -> 1/sqrt(head_dim)                                              */
+    void *pool;                 /* device; K/V store for registered packets and adapters              */
+    uint64_t pool_bytes;        /* capacity in tokens = pool_bytes / kvp_token_bytes(cfg)             */
+    void *workspace;            /* device; plans, staged rows, appended query K/V, split partials     */
+    uint64_t workspace_bytes;   /* at least kvp_workspace_bytes(cfg)                                  */
+    int32_t max_packets;
+    int32_t max_adapters;
+    int32_t max_batch;          /* requests per assembly                                              */
+    int32_t max_slots;          /* packets per assembly, summed over its requests                     */
+    int32_t max_prefix_tokens;  /* composed prefix length of one request                              */
+    int32_t max_query_tokens;   /* q_len                                                              */
+    int32_t max_ws_rows;        /* workspace K/V rows per assembly: sum over requests of
+                                   (adapter tokens + max_query_tokens), or with KVP_MATERIALIZE of
+                                   (prefix tokens + max_query_tokens)                                  */
+    int32_t max_assemblies;     /* assemblies alive at once (ring; ids older than this are dropped)   */
+} kvp_config;
+
+/* Bytes of pool one token occupies (K and V, all layers and kv heads).  0 if cfg is invalid. */
+KVP_API uint64_t kvp_token_bytes(const kvp_config *cfg);
+
+/* Workspace size the configuration needs.  0 if cfg is invalid. */
+KVP_API uint64_t kvp_workspace_bytes(const kvp_config *cfg);
+
+/*
+ * Create a context on cfg->device.  The pool and the workspace are borrowed, must be 1024-byte
+ * aligned, and are zero-filled here (stream 0, synchronised before return).  Errors: KVP_ERR_INVALID
+ * (shape/dtype/alignment), KVP_ERR_CAPACITY (workspace too small), KVP_ERR_CUDA.
+ */
+KVP_API int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out);
+
+/* Free host resources.  Device memory belongs to the caller; synchronises the device first. */
+KVP_API int32_t kvp_destroy(kvp_ctx *ctx);
+
+/*
+ * Register one packet: the per-layer K/V of a document as it was computed offline for the
+ * wrapped document (Section 3.1).  k, v: device, layout [n_layers][n_tokens][n_kv_heads][head_dim];
+ * k is post-RoPE for positions cache_pos0 + t.  The rows are copied into the pool (kv-head-major
+ * planes) on `stream`; the source may be freed once the stream has passed this point.  Pool rows are
+ * assigned densely in registration order.  In a host-only context k, v may be NULL.
+ * Errors: INVALID (n_tokens <= 0, null pointers), CAPACITY (max_packets or pool full), CUDA.
+ */
+KVP_API int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens,
+                            int32_t cache_pos0, void *stream, int32_t *packet_id);
+
+/*
+ * Register one adapter: K/V of N_h header and N_t trailer soft tokens (Section 3.1, phi = {H, T}),
+ * same layout as a packet with n_tokens = n_header / n_trailer; either count may be 0 (pointers then
+ * ignored).  Header rows are stored first, trailer rows after them.  header_pos0 / trailer_pos0 are
+ * the positions at which those keys were cached.
+ */
+KVP_API int32_t kvp_register_adapter(kvp_ctx *ctx, const void *hk, const void *hv, int32_t n_header,
+                             int32_t header_pos0, const void *tk, const void *tv, int32_t n_trailer,
+                             int32_t trailer_pos0, void *stream, int32_t *adapter_id);
+
+/*
+ * Compose a batch of requests (Section 3.2 step 4: re-align by Eq. 1, then concatenate).
+ * Request b uses slots [slot_offsets[b], slot_offsets[b+1]); slot s is  header(adapter_ids[s]) |
+ * packet_ids[s] | trailer(adapter_ids[s])  in Eq. 2 order, adapter_ids[s] = -1 for "no adapter".
+ * Positions are dense from 0; a segment cached at p0 and placed at slot offset t gets Delta = t - p0
+ * (0 for every segment when KVP_REBASE is not set).  All three index arrays are host arrays.
+ *
+ * Host work: validation, segment table, tile list, cos/sin of Delta*theta_i in double precision.
+ * Device work on `stream`: one plan upload and one gather kernel that copies + re-bases either the
+ * adapter tokens only (default: documents are read in place by kvp_query_prefill) or, with
+ * KVP_MATERIALIZE, the whole prefix into the workspace cache.
+ * prefix_len (host, [batch]) is written before return.  Errors: INVALID, NOT_FOUND, CAPACITY, CUDA.
+ */
+KVP_API int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets,
+                     const int32_t *packet_ids, const int32_t *adapter_ids, uint32_t flags,
+                     void *stream, int32_t *prefix_len, int32_t *assembly_id);
+
+/*
+ * Query prefill of one layer over an assembly (Section 3.2 step 4; Fig. 2(d)): query token i of
+ * request b attends to all prefix_len[b] composed tokens and to query tokens <= i, softmax in fp32,
+ * q head h using kv head h / (Hq/Hkv).  k_new / v_new are appended to the request's cache at rows
+ * prefix_len[b] + i (readable through kvp_export_cache).
+ *   q      device [batch][q_len][n_q_heads][head_dim]
+ *   k_new  device [batch][q_len][n_kv_heads][head_dim]   (v_new likewise)
+ *   out    device [batch][q_len][n_q_heads][head_dim]
+ *   lse    device float [batch][n_q_heads][q_len] or NULL: natural-log sum of exp(scaled scores)
+ * By default q and k_new are already rotated for positions prefix_len[b] + i; KVP_ROPE_QUERY makes
+ * the library rotate them.  Errors: INVALID, NOT_FOUND, CAPACITY (q_len > max_query_tokens),
+ * STATE (host-only context), UNSUPPORTED, CUDA.  Device-side wait timeouts are reported through
+ * kvp_status_word after the stream has been synchronised.
+ */
+KVP_API int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q,
+                          const void *k_new, const void *v_new, int32_t q_len, uint32_t flags,
+                          void *out, float *lse, void *stream);
+
+/* ---- inspection helpers (not on the hot path) -------------------------------------------------- */
+
+/*
+ * The composed sequence of request b, as host arrays (any may be NULL):
+ *   src_row [prefix_len]  pool row each composed position is read from
+ *   delta   [prefix_len]  rotation offset applied to that key
+ *   seg_table [4 * n_segments]  per segment: src_row0, length, dst_pos0, delta
+ *   n_segments  number of (non-empty) segments
+ */
+KVP_API int32_t kvp_export_plan(kvp_ctx *ctx, int32_t assembly_id, int32_t b, int32_t *src_row,
+                        int32_t *delta, int32_t *seg_table, int32_t *n_segments);
+
+/*
+ * Logical composed cache of (layer, request b): rows [0, prefix_len) re-based prefix, then the rows
+ * appended by the last kvp_query_prefill of that layer.  k_out, v_out: device,
+ * [n_rows][n_kv_heads][head_dim]; n_rows = prefix_len + n_query_rows.  k_as_f32 != 0 writes k_out as
+ * float32 (the rotation result before narrowing to the stored dtype); v_out always has the stored dtype.
+ */
+KVP_API int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32_t b,
+                         int32_t n_query_rows, void *k_out, void *v_out, int32_t k_as_f32,
+                         void *stream);
+
+/* Synchronises the device and returns the device-side status word (0 = no bounded wait ran out;
+   otherwise a code identifying the wait) in *device_status, then clears it. */
+KVP_API int32_t kvp_status_word(kvp_ctx *ctx, int32_t *device_status);
+
+/* How the last kvp_query_prefill was launched (host ints, any may be NULL): kernel kind
+   (0 = fp32 CUDA-core kernel, 1 = bf16 tcgen05 kernel), CTAs, key splits, kernels launched. */
+KVP_API int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int32_t *splits, int32_t *launches);
+
+/* Launch tuning (not needed for correctness).  key KVP_TUNE_SPLIT_TARGET_CTAS: the tcgen05 path
+   splits each request's keys until about `value` CTAs exist (0 = default, 4 per SM);
+   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic). */
+enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2 };
+KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);
+
+/* Text of the last error on this context (owned by ctx; "" if none).  With ctx == NULL: the reason
+   the last kvp_create on this thread failed. */
+KVP_API const char *kvp_last_error(kvp_ctx *ctx);
+
+/* Library version, major*10000 + minor*100 + patch. */
+KVP_API int32_t kvp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVP_H_ */

@@ -1,0 +1,255 @@
+"""ctypes binding of ``libkvp.so`` - argument marshalling only; every step of the path runs in the
+library's CUDA kernels.  Function names mirror ``include/kvp.h``.
+
+PyTorch is used here for device memory and streams only (``Context`` accepts torch tensors and
+passes their ``data_ptr()``).  There is no CPU fallback: if the shared library is missing or cannot
+be loaded, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+from . import build as _build
+
+KVP_OK = 0
+STATUS_NAMES = {0: "KVP_OK", 1: "KVP_ERR_INVALID", 2: "KVP_ERR_CAPACITY", 3: "KVP_ERR_NOT_FOUND",
+                4: "KVP_ERR_STATE", 5: "KVP_ERR_UNSUPPORTED", 6: "KVP_ERR_CUDA", 7: "KVP_ERR_TIMEOUT"}
+DTYPE_F32, DTYPE_BF16 = 0, 1
+REBASE, MATERIALIZE = 1, 2
+ROPE_QUERY, FORCE_SIMPLE = 1, 2
+TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS = 1, 2
+
+
+class KvpError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {text}")
+        self.code = code
+
+
+class kvp_config(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_int32), ("device", ctypes.c_int32), ("n_layers", ctypes.c_int32),
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("rope_pairing", ctypes.c_int32), ("rope_theta", ctypes.c_double),
+        ("inv_freq", ctypes.POINTER(ctypes.c_double)), ("softmax_scale", ctypes.c_double),
+        ("pool", ctypes.c_void_p), ("pool_bytes", ctypes.c_uint64), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_uint64), ("max_packets", ctypes.c_int32), ("max_adapters", ctypes.c_int32),
+        ("max_batch", ctypes.c_int32), ("max_slots", ctypes.c_int32), ("max_prefix_tokens", ctypes.c_int32),
+        ("max_query_tokens", ctypes.c_int32), ("max_ws_rows", ctypes.c_int32), ("max_assemblies", ctypes.c_int32),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) ``libkvp.so``; raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path) or os.environ.get("KVP_REBUILD"):
+        path = _build.build()
+    L = ctypes.CDLL(path)
+    vp, i32, u32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64
+    pi32 = ctypes.POINTER(ctypes.c_int32)
+    pcfg = ctypes.POINTER(kvp_config)
+    sig = {
+        "kvp_version": (i32, []),
+        "kvp_token_bytes": (u64, [pcfg]),
+        "kvp_workspace_bytes": (u64, [pcfg]),
+        "kvp_create": (i32, [pcfg, ctypes.POINTER(vp)]),
+        "kvp_destroy": (i32, [vp]),
+        "kvp_register_packet": (i32, [vp, vp, vp, i32, i32, vp, pi32]),
+        "kvp_register_adapter": (i32, [vp, vp, vp, i32, i32, vp, vp, i32, i32, vp, pi32]),
+        "kvp_assemble": (i32, [vp, i32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
+        "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
+        "kvp_export_plan": (i32, [vp, i32, i32, pi32, pi32, pi32, pi32]),
+        "kvp_export_cache": (i32, [vp, i32, i32, i32, i32, vp, vp, i32, vp]),
+        "kvp_status_word": (i32, [vp, pi32]),
+        "kvp_last_launch": (i32, [vp, pi32, pi32, pi32, pi32]),
+        "kvp_tune": (i32, [vp, i32, i32]),
+        "kvp_last_error": (ctypes.c_char_p, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)          # AttributeError if the library lacks a declared symbol
+        fn.restype = res
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
+            "kvp_register_packet", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
+            "kvp_export_plan", "kvp_export_cache", "kvp_status_word", "kvp_last_launch", "kvp_tune",
+            "kvp_last_error"]
+
+
+def _i32_array(xs: Sequence[int]):
+    return (ctypes.c_int32 * max(1, len(xs)))(*[int(x) for x in xs])
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return int(t.data_ptr())
+
+
+class Context:
+    """Thin object wrapper over the C calls.  ``device=-1`` makes a host-only planning context
+    (no GPU needed; nothing can be launched)."""
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: str,
+                 rope_theta: float = 10000.0, rope_pairing: int = 0, softmax_scale: float = 0.0,
+                 inv_freq: Optional[Sequence[float]] = None, pool_tokens: int = 0, max_packets: int = 64,
+                 max_adapters: int = 4, max_batch: int = 1, max_slots: int = 64, max_prefix_tokens: int = 4096,
+                 max_query_tokens: int = 128, max_ws_rows: int = 0, max_assemblies: int = 1, device: int = 0):
+        self._L = lib()
+        self._h = ctypes.c_void_p()
+        cfg = kvp_config()
+        cfg.struct_bytes = ctypes.sizeof(kvp_config)
+        cfg.device = device
+        cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
+        cfg.dtype = DTYPE_BF16 if dtype == "bf16" else DTYPE_F32
+        cfg.rope_pairing = rope_pairing
+        cfg.rope_theta = rope_theta
+        self._inv_freq = None
+        if inv_freq is not None:
+            self._inv_freq = (ctypes.c_double * (head_dim // 2))(*inv_freq)
+            cfg.inv_freq = ctypes.cast(self._inv_freq, ctypes.POINTER(ctypes.c_double))
+        cfg.softmax_scale = softmax_scale
+        cfg.max_packets, cfg.max_adapters, cfg.max_batch, cfg.max_slots = max_packets, max_adapters, max_batch, max_slots
+        cfg.max_prefix_tokens, cfg.max_query_tokens = max_prefix_tokens, max_query_tokens
+        if max_ws_rows <= 0:
+            max_ws_rows = max_batch * max_query_tokens + 64 * max_slots
+        cfg.max_ws_rows, cfg.max_assemblies = max_ws_rows, max_assemblies
+        self.dtype, self.device = dtype, device
+        self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
+        self.token_bytes = int(self._L.kvp_token_bytes(ctypes.byref(cfg)))
+        if self.token_bytes == 0:
+            raise KvpError(1, "invalid configuration")
+        self.pool = self.workspace = None
+        if device >= 0:
+            import torch
+            self._torch = torch
+            dev = torch.device(f"cuda:{device}")
+            ws_bytes = int(self._L.kvp_workspace_bytes(ctypes.byref(cfg)))
+            self.pool = torch.empty(max(1, pool_tokens) * self.token_bytes + 1024, dtype=torch.uint8, device=dev)
+            self.workspace = torch.empty(ws_bytes + 1024, dtype=torch.uint8, device=dev)
+            pa = (self.pool.data_ptr() + 1023) // 1024 * 1024
+            wa = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+            cfg.pool, cfg.pool_bytes = pa, max(1, pool_tokens) * self.token_bytes
+            cfg.workspace, cfg.workspace_bytes = wa, ws_bytes
+            self.workspace_bytes = ws_bytes
+        self.cfg = cfg
+        rc = self._L.kvp_create(ctypes.byref(cfg), ctypes.byref(self._h))
+        if rc != KVP_OK:
+            raise KvpError(rc, (self._L.kvp_last_error(None) or b"").decode())
+
+    # -- plumbing ------------------------------------------------------------------------------
+    def _check(self, rc: int):
+        if rc != KVP_OK:
+            raise KvpError(rc, (self._L.kvp_last_error(self._h) or b"").decode())
+
+    def _stream(self, stream=None):
+        if self.device < 0:
+            return None
+        if stream is None:
+            stream = self._torch.cuda.current_stream(self.device)
+        return ctypes.c_void_p(stream.cuda_stream)
+
+    def close(self):
+        if self._h:
+            self._L.kvp_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the six calls ---------------------------------------------------------------------------
+    def register_packet(self, k, v, n_tokens: int, cache_pos0: int = 0, stream=None) -> int:
+        out = ctypes.c_int32(-1)
+        self._check(self._L.kvp_register_packet(self._h, _ptr(k), _ptr(v), n_tokens, cache_pos0,
+                                                self._stream(stream), ctypes.byref(out)))
+        return out.value
+
+    def register_adapter(self, hk, hv, n_header: int, header_pos0: int, tk, tv, n_trailer: int,
+                         trailer_pos0: int, stream=None) -> int:
+        out = ctypes.c_int32(-1)
+        self._check(self._L.kvp_register_adapter(self._h, _ptr(hk), _ptr(hv), n_header, header_pos0, _ptr(tk),
+                                                 _ptr(tv), n_trailer, trailer_pos0, self._stream(stream),
+                                                 ctypes.byref(out)))
+        return out.value
+
+    def assemble(self, items: Sequence[Sequence[Tuple[int, int]]], flags: int = REBASE, stream=None):
+        """items[b] = [(packet_id, adapter_id), ...].  Returns (assembly_id, prefix_len list)."""
+        offs, pids, aids = [0], [], []
+        for it in items:
+            for pid, aid in it:
+                pids.append(pid)
+                aids.append(aid)
+            offs.append(len(pids))
+        B = len(items)
+        plen = (ctypes.c_int32 * max(1, B))()
+        aid = ctypes.c_int32(-1)
+        self._check(self._L.kvp_assemble(self._h, B, _i32_array(offs), _i32_array(pids), _i32_array(aids), flags,
+                                         self._stream(stream), plen, ctypes.byref(aid)))
+        return aid.value, [int(plen[b]) for b in range(B)]
+
+    def query_prefill(self, assembly_id: int, layer: int, q, k_new, v_new, q_len: int, out, lse=None,
+                      flags: int = 0, stream=None):
+        self._check(self._L.kvp_query_prefill(self._h, assembly_id, layer, _ptr(q), _ptr(k_new), _ptr(v_new), q_len,
+                                              flags, _ptr(out), _ptr(lse), self._stream(stream)))
+
+    # -- helpers ---------------------------------------------------------------------------------
+    def export_plan(self, assembly_id: int, b: int):
+        """(src_row [P], delta [P], seg_table [n_seg][4]) of request b as numpy int32 arrays."""
+        import numpy as np
+        nseg = ctypes.c_int32(0)
+        pi = ctypes.POINTER(ctypes.c_int32)
+        self._check(self._L.kvp_export_plan(self._h, assembly_id, b, None, None, None, ctypes.byref(nseg)))
+        segs = np.zeros((max(1, nseg.value), 4), dtype=np.int32)
+        self._check(self._L.kvp_export_plan(self._h, assembly_id, b, None, None, segs.ctypes.data_as(pi),
+                                            ctypes.byref(nseg)))
+        segs = segs[:nseg.value]
+        prefix_len = int((segs[:, 1] + segs[:, 2]).max()) if nseg.value else 0
+        src = np.zeros(max(1, prefix_len), dtype=np.int32)
+        dl = np.zeros(max(1, prefix_len), dtype=np.int32)
+        self._check(self._L.kvp_export_plan(self._h, assembly_id, b, src.ctypes.data_as(pi), dl.ctypes.data_as(pi),
+                                            None, ctypes.byref(nseg)))
+        return src[:prefix_len], dl[:prefix_len], segs
+
+    def export_cache(self, assembly_id: int, layer: int, b: int, prefix_len: int, n_query_rows: int,
+                     k_as_f32: bool = False, stream=None):
+        torch = self._torch
+        dt = torch.bfloat16 if self.dtype == "bf16" else torch.float32
+        n = prefix_len + n_query_rows
+        dev = torch.device(f"cuda:{self.device}")
+        k = torch.empty((n, self.n_kv_heads, self.head_dim), dtype=torch.float32 if k_as_f32 else dt, device=dev)
+        v = torch.empty((n, self.n_kv_heads, self.head_dim), dtype=dt, device=dev)
+        self._check(self._L.kvp_export_cache(self._h, assembly_id, layer, b, n_query_rows, _ptr(k), _ptr(v),
+                                             1 if k_as_f32 else 0, self._stream(stream)))
+        return k, v
+
+    def status_word(self) -> int:
+        w = ctypes.c_int32(0)
+        rc = self._L.kvp_status_word(self._h, ctypes.byref(w))
+        if rc not in (KVP_OK, 7):
+            self._check(rc)
+        return w.value
+
+    def last_launch(self):
+        a, b, c, d = (ctypes.c_int32() for _ in range(4))
+        self._check(self._L.kvp_last_launch(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(d)))
+        return {"kind": a.value, "ctas": b.value, "splits": c.value, "launches": d.value}
+
+    def tune(self, key: int, value: int):
+        self._check(self._L.kvp_tune(self._h, key, value))

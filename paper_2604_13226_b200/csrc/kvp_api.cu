@@ -1,0 +1,618 @@
+// C ABI + host planner of the composed-cache query-prefill library.
+//
+// The planner turns a batch of requests into (i) a segment table - header | document | trailer per
+// slot, Eq. 2 order, dense positions, Delta = slot offset - cache position (Eq. 1) - and (ii) the tile
+// list the attention kernels walk: runs of <= 128 key rows that share one rotation offset, read in
+// place from the pool (documents) or from the workspace (staged adapter rows, materialised cache).
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <map>
+
+#include "kvp_internal.h"
+
+namespace {
+
+constexpr uint64_t kAlign = 1024;
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct ws_layout {
+    uint64_t status, inv_freq, slots, slot_stride, slot_plan, slot_k, slot_v, partial_o, partial_ml, q_scratch, total;
+    uint64_t rows_bytes;
+};
+
+bool valid_cfg(const kvp_config *c)
+{
+    if (!c || c->struct_bytes != (int32_t)sizeof(kvp_config)) return false;
+    if (c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0) return false;
+    if (c->n_q_heads % c->n_kv_heads) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->dtype != KVP_DTYPE_F32 && c->dtype != KVP_DTYPE_BF16) return false;
+    if (c->rope_pairing != 0 && c->rope_pairing != 1) return false;
+    if (c->max_packets <= 0 || c->max_adapters < 0 || c->max_batch <= 0 || c->max_slots <= 0) return false;
+    if (c->max_prefix_tokens <= 0 || c->max_query_tokens <= 0 || c->max_ws_rows <= 0 || c->max_assemblies <= 0)
+        return false;
+    if (!c->inv_freq && !(c->rope_theta > 0.0)) return false;
+    return true;
+}
+
+kvp_plan_layout plan_layout(const kvp_config *c)
+{
+    kvp_plan_layout p;
+    p.max_segs = 3 * c->max_slots;
+    p.max_rope = p.max_segs + 1;
+    p.max_tiles = c->max_batch * (c->max_prefix_tokens / KVP_TILE_KEYS + 2) + c->max_slots +
+                  c->max_ws_rows / KVP_TILE_KEYS + 8;
+    p.max_chunks = c->max_ws_rows / KVP_CHUNK_ROWS + p.max_segs + 8;
+    uint64_t o = 0;
+    p.items = o;  o = round_up(o + sizeof(kvp_item) * c->max_batch, 256);
+    p.tiles = o;  o = round_up(o + sizeof(kvp_tile) * p.max_tiles, 256);
+    p.chunks = o; o = round_up(o + sizeof(kvp_chunk) * p.max_chunks, 256);
+    p.segs = o;   o = round_up(o + sizeof(kvp_seg) * p.max_segs, 256);
+    p.rope = o;   o = round_up(o + sizeof(float2) * (uint64_t)p.max_rope * (c->head_dim / 2), 256);
+    p.total = o;
+    return p;
+}
+
+ws_layout workspace_layout(const kvp_config *c)
+{
+    ws_layout w;
+    const uint64_t e = c->dtype == KVP_DTYPE_BF16 ? 2 : 4;
+    const kvp_plan_layout p = plan_layout(c);
+    uint64_t o = 0;
+    w.status = o;   o += 256;
+    w.inv_freq = o; o = round_up(o + 8 * 64, kAlign);
+    w.rows_bytes = round_up((uint64_t)c->n_layers * c->n_kv_heads * c->max_ws_rows * c->head_dim * e, kAlign);
+    w.slot_plan = 0;
+    w.slot_k = round_up(p.total, kAlign);
+    w.slot_v = w.slot_k + w.rows_bytes;
+    w.slot_stride = w.slot_v + w.rows_bytes;
+    w.slots = o;    o += w.slot_stride * c->max_assemblies;
+    w.partial_o = o;  o = round_up(o + (uint64_t)KVP_MAX_SPLIT_UNITS * KVP_TILE_ROWS * c->head_dim * 4, kAlign);
+    w.partial_ml = o; o = round_up(o + (uint64_t)KVP_MAX_SPLIT_UNITS * KVP_TILE_ROWS * 8, kAlign);
+    w.q_scratch = o;  o = round_up(o + (uint64_t)c->max_batch * c->max_query_tokens * c->n_q_heads * c->head_dim * e, kAlign);
+    w.total = o;
+    return w;
+}
+
+int32_t fail(kvp_ctx *ctx, int32_t code, const char *fmt, ...) __attribute__((format(printf, 3, 4)));
+int32_t fail(kvp_ctx *ctx, int32_t code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (ctx) ctx->err = buf;
+    return code;
+}
+
+#define KVP_CUDA(ctx, call)                                                                              \
+    do {                                                                                                 \
+        cudaError_t e_ = (call);                                                                         \
+        if (e_ != cudaSuccess) return fail(ctx, KVP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));  \
+    } while (0)
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// One K or V plane set as a 3-D bf16 tensor (head_dim, rows, layer*kv_head); box = 64 columns x 128
+// rows with the 128-byte swizzle the MMA descriptors expect; out-of-range rows read as zero.
+bool make_tensor_map(encode_tiled_fn enc, CUtensorMap *tm, void *base, int head_dim, int64_t rows, int planes)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)rows, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)rows * head_dim * 2};
+    const cuuint32_t box[3] = {64, KVP_TILE_KEYS, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+kvp_plan_dev plan_dev(const kvp_ctx *ctx, int slot)
+{
+    char *base = ctx->slot_plan_dev[slot];
+    kvp_plan_dev p;
+    p.items = reinterpret_cast<const kvp_item *>(base + ctx->pl.items);
+    p.tiles = reinterpret_cast<const kvp_tile *>(base + ctx->pl.tiles);
+    p.chunks = reinterpret_cast<const kvp_chunk *>(base + ctx->pl.chunks);
+    p.segs = reinterpret_cast<const kvp_seg *>(base + ctx->pl.segs);
+    p.rope = reinterpret_cast<const float2 *>(base + ctx->pl.rope);
+    return p;
+}
+
+int find_slot(kvp_ctx *ctx, int32_t assembly_id)
+{
+    if (assembly_id < 0) return -1;
+    const int slot = assembly_id % ctx->cfg.max_assemblies;
+    return ctx->slots[slot].id == assembly_id ? slot : -1;
+}
+
+thread_local std::string g_create_error;
+
+}  // namespace
+
+extern "C" {
+
+int32_t kvp_version(void) { return 100; }
+
+uint64_t kvp_token_bytes(const kvp_config *cfg)
+{
+    if (!valid_cfg(cfg)) return 0;
+    return 2ull * cfg->n_layers * cfg->n_kv_heads * cfg->head_dim * (cfg->dtype == KVP_DTYPE_BF16 ? 2 : 4);
+}
+
+uint64_t kvp_workspace_bytes(const kvp_config *cfg)
+{
+    if (!valid_cfg(cfg)) return 0;
+    return workspace_layout(cfg).total;
+}
+
+const char *kvp_last_error(kvp_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
+{
+    if (!out) return KVP_ERR_INVALID;
+    *out = nullptr;
+    if (!valid_cfg(cfg)) { g_create_error = "invalid configuration"; return KVP_ERR_INVALID; }
+    g_create_error.clear();
+    kvp_ctx *ctx = new kvp_ctx();
+    ctx->cfg = *cfg;
+    ctx->host_only = cfg->device < 0;
+    kvp_shape &sh = ctx->shape;
+    sh.n_layers = cfg->n_layers;
+    sh.n_q_heads = cfg->n_q_heads;
+    sh.n_kv_heads = cfg->n_kv_heads;
+    sh.head_dim = cfg->head_dim;
+    sh.group = cfg->n_q_heads / cfg->n_kv_heads;
+    sh.dtype = cfg->dtype;
+    sh.pairing = cfg->rope_pairing;
+    sh.elem_bytes = cfg->dtype == KVP_DTYPE_BF16 ? 2 : 4;
+    sh.scale = (float)(cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / sqrt((double)cfg->head_dim));
+    sh.pool_rows = (int64_t)(cfg->pool_bytes / kvp_token_bytes(cfg));
+    sh.ws_rows = cfg->max_ws_rows;
+    ctx->inv_freq.resize(cfg->head_dim / 2);
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        ctx->inv_freq[i] = cfg->inv_freq ? cfg->inv_freq[i] : pow(cfg->rope_theta, -2.0 * i / cfg->head_dim);
+    ctx->cfg.inv_freq = nullptr;
+    ctx->pl = plan_layout(cfg);
+    ctx->slots.resize(cfg->max_assemblies);
+    *out = ctx;
+    if (ctx->host_only) {
+        if (sh.pool_rows <= 0) sh.pool_rows = INT32_MAX;      // sizes only: no pool behind it
+        return KVP_OK;
+    }
+
+    const ws_layout w = workspace_layout(cfg);
+    auto bail = [&](int32_t code, const char *msg) {
+        g_create_error = msg;
+        delete ctx;
+        *out = nullptr;
+        return code;
+    };
+    if (!cfg->pool || !cfg->workspace || ((uintptr_t)cfg->pool % kAlign) || ((uintptr_t)cfg->workspace % kAlign))
+        return bail(KVP_ERR_INVALID, "pool/workspace must be non-null and 1024-byte aligned");
+    if (sh.pool_rows <= 0) return bail(KVP_ERR_CAPACITY, "pool smaller than one token");
+    if (cfg->workspace_bytes < w.total) return bail(KVP_ERR_CAPACITY, "workspace too small");
+    if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(KVP_ERR_CUDA, "cudaSetDevice failed");
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(KVP_ERR_CUDA, "no device properties");
+    ctx->sm_count = prop.multiProcessorCount;
+
+    const uint64_t plane_bytes = (uint64_t)sh.n_layers * sh.n_kv_heads * sh.pool_rows * sh.head_dim * sh.elem_bytes;
+    ctx->pool_k = (char *)cfg->pool;
+    ctx->pool_v = ctx->pool_k + plane_bytes;
+    char *ws = (char *)cfg->workspace;
+    ctx->status_dev = (int32_t *)(ws + w.status);
+    for (int a = 0; a < cfg->max_assemblies; ++a) {
+        char *s = ws + w.slots + w.slot_stride * a;
+        ctx->slot_plan_dev.push_back(s + w.slot_plan);
+        ctx->slot_k.push_back(s + w.slot_k);
+        ctx->slot_v.push_back(s + w.slot_v);
+    }
+    ctx->partial_o = (float *)(ws + w.partial_o);
+    ctx->partial_ml = (float2 *)(ws + w.partial_ml);
+    ctx->q_scratch = ws + w.q_scratch;
+
+    if (cudaMemset(cfg->pool, 0, 2 * plane_bytes) != cudaSuccess ||
+        cudaMemset(cfg->workspace, 0, w.total) != cudaSuccess ||
+        cudaMemcpy(ws + w.inv_freq, ctx->inv_freq.data(), 8 * ctx->inv_freq.size(), cudaMemcpyHostToDevice) !=
+            cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess)
+        return bail(KVP_ERR_CUDA, "clearing pool/workspace failed");
+
+    for (int a = 0; a < cfg->max_assemblies; ++a) {
+        char *h = nullptr;
+        cudaEvent_t ev;
+        if (cudaHostAlloc((void **)&h, ctx->pl.total, cudaHostAllocDefault) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess)
+            return bail(KVP_ERR_CUDA, "pinned staging allocation failed");
+        ctx->slot_plan_host.push_back(h);
+        ctx->slot_event.push_back(ev);
+    }
+
+    if (sh.dtype == KVP_DTYPE_BF16 && sh.head_dim == 128 && prop.major == 10) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess && fn &&
+            qres == cudaDriverEntryPointSuccess) {
+            encode_tiled_fn enc = (encode_tiled_fn)fn;
+            const int planes = sh.n_layers * sh.n_kv_heads;
+            bool ok = make_tensor_map(enc, &ctx->tm_pool_k, ctx->pool_k, sh.head_dim, sh.pool_rows, planes) &&
+                      make_tensor_map(enc, &ctx->tm_pool_v, ctx->pool_v, sh.head_dim, sh.pool_rows, planes);
+            ctx->tm_ws_k.resize(cfg->max_assemblies);
+            ctx->tm_ws_v.resize(cfg->max_assemblies);
+            for (int a = 0; ok && a < cfg->max_assemblies; ++a)
+                ok = make_tensor_map(enc, &ctx->tm_ws_k[a], ctx->slot_k[a], sh.head_dim, sh.ws_rows, planes) &&
+                     make_tensor_map(enc, &ctx->tm_ws_v[a], ctx->slot_v[a], sh.head_dim, sh.ws_rows, planes);
+            if (!ok) return bail(KVP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+            if (kvp_attn_sm100_prepare() != cudaSuccess) return bail(KVP_ERR_CUDA, "tcgen05 kernel attribute setup failed");
+            ctx->have_tma = true;
+        }
+    }
+    return KVP_OK;
+}
+
+int32_t kvp_destroy(kvp_ctx *ctx)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!ctx->host_only) {
+        cudaSetDevice(ctx->cfg.device);
+        cudaDeviceSynchronize();
+        for (char *h : ctx->slot_plan_host) cudaFreeHost(h);
+        for (cudaEvent_t e : ctx->slot_event) cudaEventDestroy(e);
+    }
+    delete ctx;
+    return KVP_OK;
+}
+
+static int32_t store_segment(kvp_ctx *ctx, const void *k, const void *v, int32_t n, cudaStream_t st)
+{
+    if (n == 0 || ctx->host_only) return KVP_OK;
+    const kvp_shape &sh = ctx->shape;
+    KVP_CUDA(ctx, kvp_launch_store_rows(sh, k, ctx->pool_k, sh.pool_rows, ctx->pool_rows_used, n, st));
+    KVP_CUDA(ctx, kvp_launch_store_rows(sh, v, ctx->pool_v, sh.pool_rows, ctx->pool_rows_used, n, st));
+    return KVP_OK;
+}
+
+int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens, int32_t cache_pos0,
+                            void *stream, int32_t *packet_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!packet_id || n_tokens <= 0) return fail(ctx, KVP_ERR_INVALID, "register_packet: bad arguments");
+    if (!ctx->host_only && (!k || !v)) return fail(ctx, KVP_ERR_INVALID, "register_packet: null K/V");
+    if ((int)ctx->packets.size() >= ctx->cfg.max_packets) return fail(ctx, KVP_ERR_CAPACITY, "max_packets reached");
+    if (ctx->pool_rows_used + n_tokens > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
+    const int32_t rc = store_segment(ctx, k, v, n_tokens, (cudaStream_t)stream);
+    if (rc != KVP_OK) return rc;
+    ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0});
+    ctx->pool_rows_used += n_tokens;
+    *packet_id = (int32_t)ctx->packets.size() - 1;
+    return KVP_OK;
+}
+
+int32_t kvp_register_adapter(kvp_ctx *ctx, const void *hk, const void *hv, int32_t n_header, int32_t header_pos0,
+                             const void *tk, const void *tv, int32_t n_trailer, int32_t trailer_pos0, void *stream,
+                             int32_t *adapter_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!adapter_id || n_header < 0 || n_trailer < 0) return fail(ctx, KVP_ERR_INVALID, "register_adapter: bad arguments");
+    if (!ctx->host_only && ((n_header > 0 && (!hk || !hv)) || (n_trailer > 0 && (!tk || !tv))))
+        return fail(ctx, KVP_ERR_INVALID, "register_adapter: null K/V");
+    if ((int)ctx->adapter_h.size() >= ctx->cfg.max_adapters) return fail(ctx, KVP_ERR_CAPACITY, "max_adapters reached");
+    if (ctx->pool_rows_used + n_header + n_trailer > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
+    int32_t rc = store_segment(ctx, hk, hv, n_header, (cudaStream_t)stream);
+    if (rc != KVP_OK) return rc;
+    ctx->adapter_h.push_back({(int32_t)ctx->pool_rows_used, n_header, header_pos0});
+    ctx->pool_rows_used += n_header;
+    rc = store_segment(ctx, tk, tv, n_trailer, (cudaStream_t)stream);
+    if (rc != KVP_OK) { ctx->adapter_h.pop_back(); ctx->pool_rows_used -= n_header; return rc; }
+    ctx->adapter_t.push_back({(int32_t)ctx->pool_rows_used, n_trailer, trailer_pos0});
+    ctx->pool_rows_used += n_trailer;
+    *adapter_id = (int32_t)ctx->adapter_h.size() - 1;
+    return KVP_OK;
+}
+
+int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, const int32_t *packet_ids,
+                     const int32_t *adapter_ids, uint32_t flags, void *stream, int32_t *prefix_len,
+                     int32_t *assembly_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!slot_offsets || !packet_ids || !adapter_ids || !prefix_len || !assembly_id || batch <= 0)
+        return fail(ctx, KVP_ERR_INVALID, "assemble: bad arguments");
+    if (flags & ~(uint32_t)(KVP_REBASE | KVP_MATERIALIZE)) return fail(ctx, KVP_ERR_INVALID, "assemble: unknown flags");
+    const kvp_config &cfg = ctx->cfg;
+    if (batch > cfg.max_batch) return fail(ctx, KVP_ERR_CAPACITY, "assemble: batch > max_batch");
+    if (slot_offsets[0] != 0) return fail(ctx, KVP_ERR_INVALID, "assemble: slot_offsets[0] != 0");
+    for (int b = 0; b < batch; ++b)
+        if (slot_offsets[b + 1] < slot_offsets[b]) return fail(ctx, KVP_ERR_INVALID, "assemble: slot_offsets not monotone");
+    const int n_slots = slot_offsets[batch];
+    if (n_slots > cfg.max_slots) return fail(ctx, KVP_ERR_CAPACITY, "assemble: more than max_slots slots");
+    for (int s = 0; s < n_slots; ++s) {
+        if (packet_ids[s] < 0 || packet_ids[s] >= (int)ctx->packets.size())
+            return fail(ctx, KVP_ERR_NOT_FOUND, "assemble: unknown packet id %d", packet_ids[s]);
+        if (adapter_ids[s] < -1 || adapter_ids[s] >= (int)ctx->adapter_h.size())
+            return fail(ctx, KVP_ERR_NOT_FOUND, "assemble: unknown adapter id %d", adapter_ids[s]);
+    }
+    const bool rebase = flags & KVP_REBASE, mat = flags & KVP_MATERIALIZE;
+    const int half = cfg.head_dim / 2;
+
+    kvp_assembly_host as;
+    as.flags = flags;
+    as.batch = batch;
+    std::map<int32_t, int32_t> rope_of;        // delta -> rope-table index (0 = identity)
+    std::vector<int32_t> rope_delta(1, 0);
+    rope_of[0] = 0;
+    std::vector<kvp_chunk> chunks;
+    int64_t ws_cursor = 0;
+
+    auto add_chunks = [&](int32_t src, int32_t dst, int32_t n, int32_t rope) {
+        for (int32_t o = 0; o < n; o += KVP_CHUNK_ROWS)
+            chunks.push_back({src + o, dst + o, std::min<int32_t>(KVP_CHUNK_ROWS, n - o), rope});
+    };
+    auto add_tiles = [&](int16_t src, int32_t row0, int32_t n, int32_t rope, int32_t pos0) {
+        for (int32_t o = 0; o < n; o += KVP_TILE_KEYS)
+            as.tiles.push_back({row0 + o, (int16_t)std::min<int32_t>(KVP_TILE_KEYS, n - o), src, rope, pos0 + o});
+    };
+
+    for (int b = 0; b < batch; ++b) {
+        kvp_item it;
+        memset(&it, 0, sizeof it);
+        it.seg_begin = (int32_t)as.segs.size();
+        int64_t t = 0;
+        int64_t staged = 0;
+        for (int s = slot_offsets[b]; s < slot_offsets[b + 1]; ++s) {
+            const kvp_segment_host *parts[3] = {nullptr, &ctx->packets[packet_ids[s]], nullptr};
+            if (adapter_ids[s] >= 0) {
+                parts[0] = &ctx->adapter_h[adapter_ids[s]];
+                parts[2] = &ctx->adapter_t[adapter_ids[s]];
+            }
+            for (int k = 0; k < 3; ++k) {
+                const kvp_segment_host *sg = parts[k];
+                if (!sg || sg->n == 0) continue;
+                kvp_seg e;
+                memset(&e, 0, sizeof e);
+                e.src_row0 = sg->row0;
+                e.len = sg->n;
+                e.dst_pos0 = (int32_t)t;
+                e.delta = rebase ? (int32_t)(t - sg->pos0) : 0;
+                auto f = rope_of.find(e.delta);
+                if (f == rope_of.end()) {
+                    f = rope_of.emplace(e.delta, (int32_t)rope_delta.size()).first;
+                    rope_delta.push_back(e.delta);
+                }
+                e.rope = f->second;
+                e.pad[0] = -1;                   // workspace row of a staged copy, if any
+                e.pad[1] = k;                    // 0 header, 1 document, 2 trailer
+                if (!mat && k != 1) staged += sg->n;
+                as.segs.push_back(e);
+                t += sg->n;
+            }
+        }
+        if (t > cfg.max_prefix_tokens) return fail(ctx, KVP_ERR_CAPACITY, "assemble: request %d prefix %lld > max_prefix_tokens", b, (long long)t);
+        it.seg_end = (int32_t)as.segs.size();
+        it.prefix_len = (int32_t)t;
+        prefix_len[b] = (int32_t)t;
+        it.tile_begin = (int32_t)as.tiles.size();
+        if (mat) {
+            it.cache_row0 = (int32_t)ws_cursor;
+            for (int s = it.seg_begin; s < it.seg_end; ++s) {
+                kvp_seg &e = as.segs[s];
+                add_chunks(e.src_row0, it.cache_row0 + e.dst_pos0, e.len, e.rope);
+            }
+            add_tiles(1, it.cache_row0, it.prefix_len, 0, 0);
+            it.tail_row0 = it.cache_row0 + it.prefix_len;
+            ws_cursor += (int64_t)it.prefix_len + cfg.max_query_tokens;
+        } else {
+            it.cache_row0 = -1;
+            const int32_t stage0 = (int32_t)ws_cursor;
+            int32_t so = 0;
+            for (int s = it.seg_begin; s < it.seg_end; ++s) {      // adapter tokens: staged, re-based
+                kvp_seg &e = as.segs[s];
+                if (e.pad[1] == 1) continue;
+                e.pad[0] = stage0 + so;
+                add_chunks(e.src_row0, e.pad[0], e.len, e.rope);
+                so += e.len;
+            }
+            add_tiles(1, stage0, so, 0, -1);
+            for (int s = it.seg_begin; s < it.seg_end; ++s) {      // documents: read in place
+                const kvp_seg &e = as.segs[s];
+                if (e.pad[1] == 1) add_tiles(0, e.src_row0, e.len, e.rope, e.dst_pos0);
+            }
+            it.tail_row0 = stage0 + so;
+            ws_cursor += (int64_t)so + cfg.max_query_tokens;
+        }
+        it.tile_end = (int32_t)as.tiles.size();
+        if (ws_cursor > cfg.max_ws_rows) return fail(ctx, KVP_ERR_CAPACITY, "assemble: needs more than max_ws_rows workspace rows");
+        as.items.push_back(it);
+    }
+    if ((int)as.tiles.size() > ctx->pl.max_tiles || (int)chunks.size() > ctx->pl.max_chunks ||
+        (int)rope_delta.size() > ctx->pl.max_rope || (int)as.segs.size() > ctx->pl.max_segs)
+        return fail(ctx, KVP_ERR_CAPACITY, "assemble: plan tables overflow");
+    as.n_chunks = (int32_t)chunks.size();
+    as.n_rope = (int32_t)rope_delta.size();
+
+    const int32_t id = ctx->next_assembly++;
+    const int slot = id % cfg.max_assemblies;
+    as.id = id;
+    if (!ctx->host_only) {
+        cudaStream_t st = (cudaStream_t)stream;
+        KVP_CUDA(ctx, cudaSetDevice(cfg.device));
+        KVP_CUDA(ctx, cudaEventSynchronize(ctx->slot_event[slot]));      // staging buffer free again?
+        char *h = ctx->slot_plan_host[slot];
+        memcpy(h + ctx->pl.items, as.items.data(), sizeof(kvp_item) * as.items.size());
+        memcpy(h + ctx->pl.tiles, as.tiles.data(), sizeof(kvp_tile) * as.tiles.size());
+        memcpy(h + ctx->pl.chunks, chunks.data(), sizeof(kvp_chunk) * chunks.size());
+        memcpy(h + ctx->pl.segs, as.segs.data(), sizeof(kvp_seg) * as.segs.size());
+        float2 *rt = reinterpret_cast<float2 *>(h + ctx->pl.rope);
+        for (size_t r = 0; r < rope_delta.size(); ++r)
+            for (int i = 0; i < half; ++i) {
+                const double a = (double)rope_delta[r] * ctx->inv_freq[i];      // angle in double: Delta reaches 1e5
+                rt[r * half + i] = make_float2((float)cos(a), (float)sin(a));
+            }
+        const uint64_t used = ctx->pl.rope + sizeof(float2) * rope_delta.size() * half;
+        KVP_CUDA(ctx, cudaMemcpyAsync(ctx->slot_plan_dev[slot], h, used, cudaMemcpyHostToDevice, st));
+        KVP_CUDA(ctx, cudaEventRecord(ctx->slot_event[slot], st));
+        KVP_CUDA(ctx, kvp_launch_gather(ctx->shape, plan_dev(ctx, slot), as.n_chunks, ctx->pool_k, ctx->pool_v,
+                                        ctx->slot_k[slot], ctx->slot_v[slot], st));
+    }
+    ctx->slots[slot] = std::move(as);
+    *assembly_id = id;
+    return KVP_OK;
+}
+
+int32_t kvp_export_plan(kvp_ctx *ctx, int32_t assembly_id, int32_t b, int32_t *src_row, int32_t *delta,
+                        int32_t *seg_table, int32_t *n_segments)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_plan: unknown assembly %d", assembly_id);
+    const kvp_assembly_host &as = ctx->slots[slot];
+    if (b < 0 || b >= as.batch) return fail(ctx, KVP_ERR_INVALID, "export_plan: bad request index");
+    const kvp_item &it = as.items[b];
+    if (n_segments) *n_segments = it.seg_end - it.seg_begin;
+    for (int s = it.seg_begin; s < it.seg_end; ++s) {
+        const kvp_seg &e = as.segs[s];
+        if (seg_table) {
+            int32_t *row = seg_table + 4 * (s - it.seg_begin);
+            row[0] = e.src_row0; row[1] = e.len; row[2] = e.dst_pos0; row[3] = e.delta;
+        }
+        for (int o = 0; o < e.len; ++o) {
+            if (src_row) src_row[e.dst_pos0 + o] = e.src_row0 + o;
+            if (delta) delta[e.dst_pos0 + o] = e.delta;
+        }
+    }
+    return KVP_OK;
+}
+
+int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32_t b, int32_t n_query_rows,
+                         void *k_out, void *v_out, int32_t k_as_f32, void *stream)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "export_cache: host-only context");
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_cache: unknown assembly %d", assembly_id);
+    const kvp_assembly_host &as = ctx->slots[slot];
+    if (b < 0 || b >= as.batch || layer < 0 || layer >= ctx->cfg.n_layers || !k_out || !v_out || n_query_rows < 0 ||
+        n_query_rows > ctx->cfg.max_query_tokens)
+        return fail(ctx, KVP_ERR_INVALID, "export_cache: bad arguments");
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    KVP_CUDA(ctx, kvp_launch_export(ctx->shape, plan_dev(ctx, slot), b, layer, as.items[b].prefix_len, n_query_rows,
+                                    ctx->pool_k, ctx->pool_v, ctx->slot_k[slot], ctx->slot_v[slot], k_out, v_out,
+                                    k_as_f32, (cudaStream_t)stream));
+    return KVP_OK;
+}
+
+int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
+                          const void *v_new, int32_t q_len, uint32_t flags, void *out, float *lse, void *stream)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "query_prefill: host-only context has no device to run on");
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "query_prefill: unknown assembly %d", assembly_id);
+    if (!q || !k_new || !v_new || !out || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
+        return fail(ctx, KVP_ERR_INVALID, "query_prefill: bad arguments");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    if (q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: q_len > max_query_tokens");
+    kvp_assembly_host &as = ctx->slots[slot];
+    const kvp_shape &sh = ctx->shape;
+    cudaStream_t st = (cudaStream_t)stream;
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const kvp_plan_dev plan = plan_dev(ctx, slot);
+    const int rope_query = (flags & KVP_ROPE_QUERY) ? 1 : 0;
+    const double *inv_freq_dev = reinterpret_cast<const double *>((char *)ctx->cfg.workspace + 256);
+
+    int launches = 0;
+    KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
+                                    layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
+    ++launches;
+    const void *q_used = rope_query ? (const void *)ctx->q_scratch : q;
+    as.last_q_len = q_len;
+
+    const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
+    int32_t ctas = 0, splits = 1;
+    if (!fast) {
+        KVP_CUDA(ctx, kvp_launch_attn_simple(sh, plan, as.batch, q_len, layer, q_used, ctx->pool_k, ctx->pool_v,
+                                             ctx->slot_k[slot], ctx->slot_v[slot], out, lse, &ctas, st));
+        ++launches;
+        ctx->last_kind = 0;
+    } else {
+        const int n_mtiles = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
+        const int units = as.batch * sh.n_kv_heads * n_mtiles;
+        int min_tiles = INT32_MAX;
+        for (const kvp_item &it : as.items) min_tiles = std::min(min_tiles, it.tile_end - it.tile_begin + 1);
+        const int target = ctx->split_target_ctas > 0 ? ctx->split_target_ctas : 4 * ctx->sm_count;
+        if (units < target) {
+            splits = (target + units - 1) / units;
+            splits = std::min(splits, std::max(1, min_tiles / 4));
+            splits = std::min(splits, KVP_MAX_SPLIT_UNITS / units);
+            splits = std::max(splits, 1);
+        }
+        if (ctx->force_splits > 0) splits = std::min(ctx->force_splits, std::max(1, KVP_MAX_SPLIT_UNITS / units));
+        kvp_attn_sm100_args a;
+        a.plan = plan;
+        a.batch = as.batch;
+        a.q_len = q_len;
+        a.layer = layer;
+        a.n_splits = splits;
+        a.n_mtiles = n_mtiles;
+        a.q = q_used;
+        a.out = out;
+        a.lse = lse;
+        a.partial_o = ctx->partial_o;
+        a.partial_ml = ctx->partial_ml;
+        a.status = ctx->status_dev;
+        KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot],
+                                            ctx->tm_ws_v[slot], &ctas, st));
+        ++launches;
+        if (splits > 1) {
+            KVP_CUDA(ctx, kvp_launch_merge(sh, as.batch, q_len, splits, n_mtiles, ctx->partial_o, ctx->partial_ml, out,
+                                           lse, st));
+            ++launches;
+        }
+        ctx->last_kind = 1;
+    }
+    ctx->last_ctas = ctas;
+    ctx->last_splits = splits;
+    ctx->last_launches = launches;
+    return KVP_OK;
+}
+
+int32_t kvp_status_word(kvp_ctx *ctx, int32_t *device_status)
+{
+    if (!ctx || !device_status) return KVP_ERR_INVALID;
+    if (ctx->host_only) { *device_status = 0; return KVP_OK; }
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    KVP_CUDA(ctx, cudaDeviceSynchronize());
+    KVP_CUDA(ctx, cudaMemcpy(device_status, ctx->status_dev, 4, cudaMemcpyDeviceToHost));
+    if (*device_status != 0) {
+        KVP_CUDA(ctx, cudaMemset(ctx->status_dev, 0, 4));
+        return fail(ctx, KVP_ERR_TIMEOUT, "device-side bounded wait ran out (code %d)", *device_status);
+    }
+    return KVP_OK;
+}
+
+int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int32_t *splits, int32_t *launches)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (kind) *kind = ctx->last_kind;
+    if (ctas) *ctas = ctx->last_ctas;
+    if (splits) *splits = ctx->last_splits;
+    if (launches) *launches = ctx->last_launches;
+    return KVP_OK;
+}
+
+int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (key == KVP_TUNE_SPLIT_TARGET_CTAS) ctx->split_target_ctas = value;
+    else if (key == KVP_TUNE_FORCE_SPLITS) ctx->force_splits = value;
+    else return fail(ctx, KVP_ERR_INVALID, "tune: unknown key %d", key);
+    return KVP_OK;
+}
+
+}  // extern "C"

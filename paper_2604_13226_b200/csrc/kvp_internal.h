@@ -1,0 +1,162 @@
+// Internal declarations shared by the host planner and the CUDA kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/kvp.h"
+
+#define KVP_TILE_KEYS 128      // keys per attention tile (one TMA box of K or V rows)
+#define KVP_TILE_ROWS 128      // packed query rows per CTA tile (MMA M)
+#define KVP_CHUNK_ROWS 32      // rows per gather work item
+#define KVP_MAX_SPLIT_UNITS 2048
+
+// ---- device-visible plan records (written by the host planner, uploaded once per assembly) -----
+
+struct kvp_tile {              // one run of <= 128 consecutive key rows sharing one rotation offset
+    int32_t row0;              // first row, in the pool (src 0) or in the workspace rows (src 1)
+    int16_t n_keys;            // 1..128
+    int16_t src;               // 0 pool, 1 workspace
+    int32_t rope;              // rope-table index of the offset still to be applied to these keys (0 = none)
+    int32_t pos0;              // composed position of the first key (diagnostics)
+};
+
+struct kvp_chunk {             // gather work item: <= 32 rows copied pool -> workspace, keys rotated
+    int32_t src_row0;
+    int32_t dst_row0;
+    int32_t n_rows;
+    int32_t rope;              // rope-table index (0 = identity: byte copy)
+};
+
+struct kvp_seg {               // one segment of a composed request (header, document or trailer)
+    int32_t src_row0;
+    int32_t len;
+    int32_t dst_pos0;
+    int32_t delta;
+    int32_t rope;
+    int32_t pad[3];
+};
+
+struct kvp_item {              // one request of the batch
+    int32_t prefix_len;
+    int32_t tile_begin, tile_end;      // its prefix tiles in the tile array
+    int32_t seg_begin, seg_end;        // its segments
+    int32_t tail_row0;                 // workspace row where its query K/V rows are appended
+    int32_t cache_row0;                // workspace row of composed position 0 (materialised), else -1
+    int32_t pad;
+};
+
+// Offsets (bytes) of the arrays inside one plan blob; identical on host and device.
+struct kvp_plan_layout {
+    uint64_t items, tiles, chunks, segs, rope, total;
+    int32_t max_tiles, max_chunks, max_segs, max_rope;
+};
+
+// Pointers into a device-resident plan, passed to kernels by value.
+struct kvp_plan_dev {
+    const kvp_item *items;
+    const kvp_tile *tiles;
+    const kvp_chunk *chunks;
+    const kvp_seg *segs;
+    const float2 *rope;        // [n_rope][head_dim/2] (cos, sin) of delta * theta_i
+};
+
+struct kvp_shape {
+    int32_t n_layers, n_q_heads, n_kv_heads, head_dim, group, dtype, pairing, elem_bytes;
+    float scale;               // softmax scale
+    int64_t pool_rows;         // rows per (layer, kv head) plane in the pool
+    int64_t ws_rows;           // rows per plane in one assembly's workspace rows
+};
+
+// ---- host-side context -----------------------------------------------------------------------
+
+struct kvp_segment_host { int32_t row0, n, pos0; };
+
+struct kvp_assembly_host {
+    int32_t id = -1;
+    uint32_t flags = 0;
+    int32_t batch = 0;
+    std::vector<kvp_item> items;
+    std::vector<kvp_seg> segs;
+    std::vector<kvp_tile> tiles;
+    int32_t n_chunks = 0, n_rope = 0;
+    int32_t last_q_len = 0;
+};
+
+struct kvp_ctx {
+    kvp_config cfg;
+    kvp_shape shape;
+    bool host_only = false;
+    std::vector<double> inv_freq;
+    std::vector<kvp_segment_host> packets;
+    std::vector<kvp_segment_host> adapter_h, adapter_t;
+    int64_t pool_rows_used = 0;
+
+    // device memory carved out of the caller's buffers
+    char *pool_k = nullptr, *pool_v = nullptr;
+    int32_t *status_dev = nullptr;
+    kvp_plan_layout pl;
+    std::vector<char *> slot_plan_dev;     // per assembly slot
+    std::vector<char *> slot_k, slot_v;    // per assembly slot: workspace rows
+    float *partial_o = nullptr;            // [units][128][head_dim]
+    float2 *partial_ml = nullptr;          // [units][128] (running max, running sum)
+    char *q_scratch = nullptr;
+    float2 *q_rope = nullptr;              // [max_batch*max_query][head_dim/2] for KVP_ROPE_QUERY
+
+    // pinned host staging (one per slot) and the event guarding its reuse
+    std::vector<char *> slot_plan_host;
+    std::vector<cudaEvent_t> slot_event;
+    std::vector<kvp_assembly_host> slots;
+    int32_t next_assembly = 0;
+
+    // TMA descriptors (bf16, head_dim 128 only)
+    bool have_tma = false;
+    CUtensorMap tm_pool_k, tm_pool_v;
+    std::vector<CUtensorMap> tm_ws_k, tm_ws_v;
+
+    int32_t sm_count = 148;
+    int32_t split_target_ctas = 0, force_splits = 0;
+    int32_t last_kind = -1, last_ctas = 0, last_splits = 0, last_launches = 0;
+    std::string err;
+};
+
+// ---- kernel launchers (kvp_kernels.cu, kvp_attn_sm100.cu) ---------------------------------------
+
+cudaError_t kvp_launch_store_rows(const kvp_shape &sh, const void *src, char *dst_plane0, int64_t plane_rows,
+                                  int64_t dst_row0, int32_t n_tokens, cudaStream_t st);
+cudaError_t kvp_launch_gather(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t n_chunks,
+                              const char *pool_k, const char *pool_v, char *ws_k, char *ws_v, cudaStream_t st);
+cudaError_t kvp_launch_append(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
+                              const void *q, const void *k_new, const void *v_new, char *ws_k, char *ws_v,
+                              int32_t layer, int32_t rope_query, const double *inv_freq_dev, void *q_rot,
+                              cudaStream_t st);
+cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t b, int32_t layer,
+                              int32_t prefix_len, int32_t n_query_rows, const char *pool_k, const char *pool_v,
+                              const char *ws_k, const char *ws_v, void *k_out, void *v_out, int32_t k_as_f32,
+                              cudaStream_t st);
+cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
+                                   int32_t layer, const void *q, const char *pool_k, const char *pool_v,
+                                   const char *ws_k, const char *ws_v, void *out, float *lse, int32_t *ctas,
+                                   cudaStream_t st);
+
+struct kvp_attn_sm100_args {
+    kvp_plan_dev plan;
+    int32_t batch, q_len, layer, n_splits, n_mtiles;
+    const void *q;
+    void *out;
+    float *lse;
+    float *partial_o;
+    float2 *partial_ml;
+    int32_t *status;
+};
+cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn_sm100_args &a, const CUtensorMap &tm_pool_k,
+                                  const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
+                                  const CUtensorMap &tm_ws_v, int32_t *ctas, cudaStream_t st);
+cudaError_t kvp_launch_merge(const kvp_shape &sh, int32_t batch, int32_t q_len, int32_t n_splits, int32_t n_mtiles,
+                             const float *partial_o, const float2 *partial_ml, void *out, float *lse,
+                             cudaStream_t st);
+cudaError_t kvp_attn_sm100_prepare(void);

@@ -1,0 +1,223 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Integer/byte work must be bit-exact; fp32 re-basing within 1e-4 relative per rotated
+pair; bf16 attention within max-abs 2e-2 and mean-abs 2e-3; fp32 attention within 2e-5 (derived:
+fp32 dot products of <= 128 terms and online-softmax rescaling give ~1e-6 relative on O(1) values)."""
+import numpy as np
+import pytest
+
+from oracle import reference as orc
+from paper_2604_13226_b200 import binding as kvp
+from paper_2604_13226_b200 import inputs as gen
+from paper_2604_13226_b200.session import Session, torch_to_np
+from helpers import make_store, oracle_outputs
+
+pytestmark = pytest.mark.gpu
+
+BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
+F32_MAX_ABS = 2e-5
+
+
+def pair_rel_err(k_gpu, k_ref, pairing):
+    """max over pairs of |gpu - ref|_inf / |ref pair|_2 (rotation-invariant relative error)."""
+    d = k_ref.shape[-1]
+    if pairing == 0:
+        a, b, ga, gb = k_ref[..., : d // 2], k_ref[..., d // 2:], k_gpu[..., : d // 2], k_gpu[..., d // 2:]
+    else:
+        a, b, ga, gb = k_ref[..., 0::2], k_ref[..., 1::2], k_gpu[..., 0::2], k_gpu[..., 1::2]
+    nrm = np.sqrt(a * a + b * b)
+    err = np.maximum(np.abs(ga - a), np.abs(gb - b))
+    return float(np.max(err / np.maximum(nrm, 1e-30)))
+
+
+def check_attention(wl, sess, layer=0, flags=0, rope_query=False, rows_subset=None):
+    out, lse = sess.prefill(layer, flags | (kvp.ROPE_QUERY if rope_query else 0))
+    assert sess.ctx.status_word() == 0
+    s = wl.shape
+    o = orc.widen(torch_to_np(out, s.dtype), s.dtype)          # [B][Lq][Hq][d]
+    lse = lse.cpu().numpy().astype(np.float64)                  # [B][Hq][Lq]
+    ref = oracle_outputs(wl, layer, rope_query=rope_query)
+    worst = 0.0
+    for b in range(wl.batch):
+        ro, rl = ref[b][0], ref[b][1]
+        ro = ro.reshape(wl.q_len, s.n_q_heads, s.head_dim)
+        rl = rl.reshape(wl.q_len, s.n_q_heads).T
+        err = np.abs(o[b] - ro)
+        if s.dtype == "bf16":
+            assert err.max() <= BF16_MAX_ABS, (b, err.max())
+            assert err.mean() <= BF16_MEAN_ABS, (b, err.mean())
+            assert np.max(np.abs(lse[b] - rl)) <= 2e-2
+        else:
+            assert err.max() <= F32_MAX_ABS, (b, err.max())
+            assert np.max(np.abs(lse[b] - rl)) <= 1e-4
+        worst = max(worst, err.max())
+    return worst
+
+
+# ------------------------------------------------------------------------------------------------
+# assembly / gather / re-basing
+# ------------------------------------------------------------------------------------------------
+
+def ragged_small(dtype="bf16", d=128, pairing=0, seed=3):
+    shape = gen.ModelShape(2, 8, 2, d, dtype, 500000.0, pairing)
+    lens = [200, 37, 300, 129]
+    items = [[(0, 0), (2, 0), (1, -1)], [(3, 0), (0, 0)]]
+    return gen.make_workload(shape, lens, items, q_len=40, n_header=16, n_trailer=16, seed=seed,
+                             packet_pos0=[0, 3, 0, 1000])
+
+
+@pytest.mark.parametrize("materialize", [False, True])
+@pytest.mark.parametrize("maker", [gen.config1, gen.config2, ragged_small,
+                                   lambda: ragged_small("f32", 64, 1), lambda: ragged_small("bf16", 128, 1)])
+def test_index_map_and_cache_bytes(maker, materialize):
+    wl = maker()
+    s = wl.shape
+    sess = Session(wl, materialize=materialize)
+    pool_before = sess.ctx.pool.clone()
+    st = make_store(wl)
+    f = orc.inv_freq(s.rope_theta, s.head_dim)
+    for rebase in (True, False):
+        aid, plen = sess.assemble(rebase=rebase)
+        for b in range(wl.batch):
+            plan = orc.compose(st, wl.items[b], rebase)
+            src, dl, segs = sess.ctx.export_plan(aid, b)
+            assert plen[b] == plan.prefix_len
+            assert np.array_equal(src, plan.src_row) and np.array_equal(dl, plan.delta)
+            assert np.array_equal(segs, plan.segments)
+            for layer in range(s.n_layers):
+                k_ref, v_ref, k_raw = orc.composed_kv(st, plan, layer, f, s.rope_pairing)
+                k32, v = sess.ctx.export_cache(aid, layer, b, plen[b], 0, k_as_f32=True)
+                kst, _ = sess.ctx.export_cache(aid, layer, b, plen[b], 0, k_as_f32=False)
+                v = orc.widen(torch_to_np(v, s.dtype), s.dtype)
+                assert np.array_equal(v, v_ref)                             # copied bytes: bit-exact
+                kst = orc.widen(torch_to_np(kst, s.dtype), s.dtype)
+                if not rebase:
+                    assert np.array_equal(kst, k_raw)                       # no rotation: bit-exact
+                else:
+                    k32 = k32.cpu().numpy().astype(np.float64)
+                    if s.dtype == "f32" or not materialize:
+                        # the fp32 rotation result itself (before any narrowing) where it is observable
+                        staged = np.zeros(plen[b], dtype=bool)
+                        for (kind, _), (r0, n, dst, dlt) in zip(plan.refs, plan.segments):
+                            if kind != "packet":
+                                staged[dst:dst + n] = True
+                        sel = ~staged if s.dtype == "bf16" else np.ones(plen[b], dtype=bool)
+                        if sel.any():
+                            assert pair_rel_err(k32[sel], k_ref[sel], s.rope_pairing) <= 1e-4
+                    # stored dtype: within half a bf16 ulp (2^-9 relative) of the oracle, pairwise
+                    tol = 1e-4 if s.dtype == "f32" else 2.0 ** -8
+                    assert pair_rel_err(kst, k_ref, s.rope_pairing) <= tol
+    assert bool((sess.ctx.pool == pool_before).all())                       # packets are immutable
+    assert sess.ctx.status_word() == 0
+    sess.close()
+
+
+def test_large_delta_rotation_accuracy():
+    # offsets of ~130K positions: the angle must be formed in double precision
+    shape = gen.ModelShape(1, 8, 2, 128, "f32", 500000.0, 0)
+    wl = gen.make_workload(shape, [64, 64], [[(0, 0), (1, 0)]], q_len=8, seed=5, packet_pos0=[-131000, 7],
+                           adapter_pos0=[(-99999, 50000)])
+    sess = Session(wl, materialize=True)
+    aid, plen = sess.assemble()
+    st = make_store(wl)
+    plan = orc.compose(st, wl.items[0])
+    assert np.abs(plan.delta).max() > 130000
+    k_ref, v_ref, _ = orc.composed_kv(st, plan, 0, orc.inv_freq(shape.rope_theta, 128))
+    k32, _ = sess.ctx.export_cache(aid, 0, 0, plen[0], 0, k_as_f32=True)
+    assert pair_rel_err(k32.cpu().numpy().astype(np.float64), k_ref, 0) <= 1e-4
+    sess.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# attention
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("materialize", [False, True])
+def test_config1_fp32(materialize):
+    wl = gen.config1()
+    sess = Session(wl, materialize=materialize)
+    sess.assemble()
+    check_attention(wl, sess)
+    assert sess.ctx.last_launch()["kind"] == 0
+    # appended query K/V land behind the prefix
+    k, v = sess.ctx.export_cache(sess.assembly_id, 0, 0, sess.prefix_len[0], wl.q_len)
+    assert np.array_equal(k.cpu().numpy()[sess.prefix_len[0]:], wl.k_new[0][0])
+    assert np.array_equal(v.cpu().numpy()[sess.prefix_len[0]:], wl.v_new[0][0])
+    sess.close()
+
+
+@pytest.mark.parametrize("materialize", [False, True])
+@pytest.mark.parametrize("simple", [False, True])
+def test_config2_bf16(materialize, simple):
+    wl = gen.config2()
+    sess = Session(wl, materialize=materialize)
+    sess.assemble()
+    check_attention(wl, sess, flags=kvp.FORCE_SIMPLE if simple else 0)
+    assert sess.ctx.last_launch()["kind"] == (0 if simple else 1)
+    sess.close()
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+def test_config2_forced_splits(splits):
+    wl = gen.config2()
+    sess = Session(wl)
+    sess.assemble()
+    sess.ctx.tune(kvp.TUNE_FORCE_SPLITS, splits)
+    check_attention(wl, sess)
+    assert sess.ctx.last_launch()["splits"] == splits
+    sess.close()
+
+
+@pytest.mark.parametrize("pairing", [0, 1])
+@pytest.mark.parametrize("materialize", [False, True])
+def test_ragged_batch_bf16(pairing, materialize):
+    wl = ragged_small("bf16", 128, pairing)
+    sess = Session(wl, materialize=materialize)
+    sess.assemble()
+    for layer in range(wl.shape.n_layers):
+        check_attention(wl, sess, layer=layer)
+    sess.close()
+
+
+def test_qwen_like_group7_long_query():
+    # g = 7 (rows of one token straddle MMA tiles), q_len 300 (three causal key tiles, 17 row tiles)
+    shape = gen.ModelShape(1, 28, 4, 128, "bf16", 1000000.0, 0)
+    lens = [256, 700, 1024, 333]
+    wl = gen.make_workload(shape, lens, [[(0, 0), (1, 0)], [(2, 0), (3, 0), (0, 0)]], q_len=300, seed=8,
+                           outlier_channels=2)
+    sess = Session(wl)
+    sess.assemble()
+    check_attention(wl, sess)
+    sess.ctx.tune(kvp.TUNE_FORCE_SPLITS, 4)
+    check_attention(wl, sess)
+    sess.close()
+
+
+def test_rope_query_flag():
+    for wl in (gen.config1(), ragged_small()):
+        sess = Session(wl)
+        sess.assemble()
+        check_attention(wl, sess, rope_query=True)
+        sess.close()
+
+
+def test_no_adapters_no_rebase_and_single_tiny_packet():
+    shape = gen.ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
+    wl = gen.make_workload(shape, [1, 130], [[(0, -1)], [(1, -1), (0, -1)]], q_len=1, n_header=0, n_trailer=0, seed=9,
+                           rebase=False)
+    sess = Session(wl)
+    sess.assemble()
+    check_attention(wl, sess)
+    sess.close()
+
+
+def test_short_query_many_splits_and_tensor_vs_simple_kernel():
+    shape = gen.ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
+    wl = gen.make_workload(shape, [2048] * 4, [[(p, 0) for p in range(4)]], q_len=16, seed=10)
+    sess = Session(wl)
+    sess.assemble()
+    check_attention(wl, sess)
+    assert sess.ctx.last_launch()["splits"] > 1
+    a, _ = sess.prefill(0)
+    b, _ = sess.prefill(0, kvp.FORCE_SIMPLE)
+    assert float((a.float() - b.float()).abs().max()) <= 2e-2
+    sess.close()

@@ -1,0 +1,130 @@
+"""CPU-side checks of the product library: it loads, exports what the header declares, validates
+arguments on the host, and its planner's index map equals the oracle's composition bit for bit."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import reference as orc
+from paper_2604_13226_b200 import binding as kvp
+from paper_2604_13226_b200 import inputs as gen
+from helpers import make_store
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "kvp.h")).read()
+    declared = sorted(set(re.findall(r"KVP_API[^;(]*?\b(kvp_\w+)\s*\(", header)))
+    assert len(declared) >= 12 and "kvp_query_prefill" in declared and "kvp_assemble" in declared
+    L = kvp.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(kvp.EXPORTED) == declared
+    assert L.kvp_version() >= 100
+
+
+def host_ctx(shape, wl, **kw):
+    n_slots = sum(len(it) for it in wl.items)
+    args = dict(max_packets=max(1, len(wl.packets)), max_adapters=max(1, len(wl.adapters)), max_batch=wl.batch,
+                max_slots=max(1, n_slots), max_prefix_tokens=max(wl.prefix_len(b) for b in range(wl.batch)),
+                max_query_tokens=wl.q_len, max_ws_rows=sum(wl.prefix_len(b) for b in range(wl.batch)) + wl.batch * wl.q_len,
+                device=-1)
+    args.update(kw)
+    ctx = kvp.Context(shape.n_layers, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.dtype,
+                      rope_theta=shape.rope_theta, **args)
+    for p in wl.packets:
+        ctx.register_packet(None, None, p.n_tokens, p.cache_pos0)
+    for a in wl.adapters:
+        ctx.register_adapter(None, None, a.n_header, a.header_pos0, None, None, a.n_trailer, a.trailer_pos0)
+    return ctx
+
+
+def ragged_workload(seed=0):
+    shape = gen.ModelShape(2, 4, 2, 64, "bf16", 10000.0)
+    lens = [37, 128, 300, 1, 129, 64]
+    items = [[(0, 0), (2, 1), (5, -1)], [(3, 1)], [(4, 0), (1, 0), (0, 1), (2, -1)]]
+    return gen.make_workload(shape, lens, items, q_len=5, n_header=3, n_trailer=2, n_adapters=2, seed=seed,
+                             packet_pos0=[0, 5, 0, 7, 100, 0], adapter_pos0=[(0, 0), (2, 40)])
+
+
+@pytest.mark.parametrize("flags", [kvp.REBASE, 0, kvp.REBASE | kvp.MATERIALIZE])
+def test_planner_index_map_equals_oracle(flags):
+    wl = ragged_workload()
+    ctx = host_ctx(wl.shape, wl)
+    aid, plen = ctx.assemble(wl.items, flags)
+    st = make_store(wl)
+    for b, slots in enumerate(wl.items):
+        plan = orc.compose(st, slots, rebase=bool(flags & kvp.REBASE))
+        assert plen[b] == plan.prefix_len == wl.prefix_len(b)
+        src, dl, segs = ctx.export_plan(aid, b)
+        assert np.array_equal(src, plan.src_row)
+        assert np.array_equal(dl, plan.delta)
+        assert np.array_equal(segs, plan.segments)
+    ctx.close()
+
+
+def test_planner_config1_and_config2_layouts():
+    for wl in (gen.config1(), gen.config2()):
+        ctx = host_ctx(wl.shape, wl)
+        aid, plen = ctx.assemble(wl.items, kvp.REBASE)
+        plan = orc.compose(make_store(wl), wl.items[0])
+        src, dl, segs = ctx.export_plan(aid, 0)
+        assert plen[0] == plan.prefix_len
+        assert np.array_equal(src, plan.src_row) and np.array_equal(dl, plan.delta) and np.array_equal(segs, plan.segments)
+        ctx.close()
+
+
+def test_argument_errors_are_status_codes():
+    wl = ragged_workload()
+    ctx = host_ctx(wl.shape, wl, max_slots=8)
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.assemble([[(99, 0)]])
+    assert e.value.code == 3
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.assemble([[(0, 7)]])
+    assert e.value.code == 3
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.assemble([[(0, 0)] * 9])
+    assert e.value.code == 2                       # more slots than max_slots
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.assemble([[(2, 0)] * 8])
+    assert e.value.code == 2                       # prefix longer than max_prefix_tokens
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.assemble(wl.items, 64)
+    assert e.value.code == 1                       # unknown flag
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.register_packet(None, None, 0, 0)
+    assert e.value.code == 1
+    aid, plen = ctx.assemble(wl.items)
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.export_plan(aid + 5, 0)
+    assert e.value.code == 3
+    # a host-only context cannot launch anything: the call fails loudly instead of computing on the CPU
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.query_prefill(aid, 0, 1, 1, 1, 1, 1)
+    assert e.value.code == 4
+    ctx.close()
+
+
+def test_bad_configurations_rejected():
+    for kw in (dict(n_q_heads=5, n_kv_heads=2), dict(head_dim=96), dict(n_layers=0)):
+        args = dict(n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64)
+        args.update(kw)
+        with pytest.raises(kvp.KvpError):
+            kvp.Context(args["n_layers"], args["n_q_heads"], args["n_kv_heads"], args["head_dim"], "bf16", device=-1)
+
+
+def test_assembly_ring_drops_old_ids():
+    wl = ragged_workload()
+    ctx = host_ctx(wl.shape, wl, max_assemblies=2)
+    a0, plen = ctx.assemble(wl.items)
+    a1, _ = ctx.assemble(wl.items)
+    a2, _ = ctx.assemble(wl.items)
+    assert (a0, a1, a2) == (0, 1, 2)
+    ctx.export_plan(a1, 0)
+    ctx.export_plan(a2, 0)
+    with pytest.raises(kvp.KvpError):
+        ctx.export_plan(a0, 0)
+    ctx.close()
