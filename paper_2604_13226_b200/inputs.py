@@ -217,8 +217,10 @@ def make_workload(shape: ModelShape,
     q = to_stored(rng.standard_normal((L, B, q_len, Hq, d), dtype=np.float32), shape.dtype)
     k_new = to_stored(rng.standard_normal((L, B, q_len, Hkv, d), dtype=np.float32), shape.dtype)
     v_new = to_stored(rng.standard_normal((L, B, q_len, Hkv, d), dtype=np.float32), shape.dtype)
-    return Workload(shape, packets, adapters, [list(map(tuple, it)) for it in items], q, k_new, v_new,
-                    rebase=rebase, name=name, seed=seed)
+    wl = Workload(shape, packets, adapters, [list(map(tuple, it)) for it in items], q, k_new, v_new,
+                  rebase=rebase, name=name, seed=seed)
+    wl.notes["chan_scale"] = chan_scale        # [L][1][Hkv][d] multipliers applied to packet K/V, or None
+    return wl
 
 
 def config1(seed: int = 0) -> Workload:
@@ -313,6 +315,7 @@ class DeviceWorkload:
         self.name = spec.name
         self._base = spec.seed * 1_000_003
         self._chan = None
+        self.notes = {"chan_scale": None}
         if spec.outlier_channels > 0:
             s = spec.shape
             crng = np.random.default_rng(spec.seed + 7919)
@@ -321,6 +324,7 @@ class DeviceWorkload:
                 for h in range(s.n_kv_heads):
                     cs[l, 0, h, crng.choice(s.head_dim, size=spec.outlier_channels, replace=False)] = spec.outlier_scale
             self._chan = torch.from_numpy(cs).to(self.device)
+            self.notes["chan_scale"] = cs
 
     @property
     def batch(self) -> int:

@@ -1,7 +1,10 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
 seeded inputs.  Integer/byte work must be bit-exact; fp32 re-basing within 1e-4 relative per rotated
 pair; bf16 attention within max-abs 2e-2 and mean-abs 2e-3; fp32 attention within 2e-5 (derived:
-fp32 dot products of <= 128 terms and online-softmax rescaling give ~1e-6 relative on O(1) values)."""
+fp32 dot products of <= 128 terms and online-softmax rescaling give ~1e-6 relative on O(1) values).
+The absolute bounds are for unit-scale values: the output is linear in V, so a value channel that
+the workload multiplies by 8 ("outlier channel") carries 8x the value, 8x the bf16 rounding of the
+output and of the probabilities, and therefore 8x the bound."""
 import numpy as np
 import pytest
 
@@ -42,6 +45,9 @@ def check_attention(wl, sess, layer=0, flags=0, rope_query=False, rows_subset=No
         ro = ro.reshape(wl.q_len, s.n_q_heads, s.head_dim)
         rl = rl.reshape(wl.q_len, s.n_q_heads).T
         err = np.abs(o[b] - ro)
+        cs = wl.notes.get("chan_scale")
+        if cs is not None:                                       # [L][1][Hkv][d] -> per (q head, channel)
+            err = err / np.repeat(cs[layer, 0], s.group, axis=0)[None, :, :]
         if s.dtype == "bf16":
             assert err.max() <= BF16_MAX_ABS, (b, err.max())
             assert err.mean() <= BF16_MEAN_ABS, (b, err.mean())
