@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of composed-cache query prefill (KV Packet serving path) on B200.
+
+A *step* is one pass of the whole hot path over one batch: ``kvp_assemble`` (plan upload + staging
+gather) followed by ``kvp_query_prefill`` for every layer, back to back on one stream.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+prints ONE JSON line.  ``value`` = query tokens/s of the whole job (batch * q_len tokens through the
+full layer stack per step), inputs resident in HBM.  ``e2e`` = the same with the step's Q/K_new/V_new
+coming from pinned host buffers and the outputs read back, copies inside the timed region.
+``roofline`` is for the dominant kernel (the tcgen05 attention kernel), its duration measured live
+with CUDA events on the launching stream.  ``cpu_baseline`` is the fp64 oracle on the host cores on a
+bounded sample.  ``--impl reference`` times that oracle as the reference arm.
+
+Workloads (seeded, synthetic, shaped like the paper's Llama-3.1-8B / Qwen2.5-7B RAG requests):
+config3 (default; Llama-3.1-8B 32-layer stack, 10 x 1024-token packets, 128 query tokens, batch 4),
+config2, config4, config5:<packets>:<q_len>:<batch>.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def make_spec(name: str, seed: int):
+    from paper_2604_13226_b200 import inputs as gen
+    if name == "config3":
+        return gen.spec_config3(seed=seed)
+    if name == "config4":
+        return gen.spec_config4(seed=seed)
+    if name == "config2":
+        s = gen.spec_config3(seed=seed, n_layers=1, batch=1, pool=5, per_item=5, doc_len=512, q_len=64)
+        s.name = "config2"
+        return s
+    if name.startswith("config5"):
+        _, n, q, b = name.split(":")
+        return gen.spec_config5(int(n), int(q), int(b), seed=seed)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_work(spec):
+    """Per layer: flops = 4 d Hq Lq (P + (Lq+1)/2) per request; bytes = prefix K,V once + Q, O, K_new,
+    V_new read and appended ('algorithmic work')."""
+    s = spec.shape
+    d, Hq, Hkv, e, Lq = s.head_dim, s.n_q_heads, s.n_kv_heads, s.elem_bytes, spec.q_len
+    flops = bytes_ = 0.0
+    for b in range(spec.batch):
+        P = spec.prefix_len(b)
+        flops += 4.0 * d * Hq * Lq * (P + (Lq + 1) / 2.0)
+        bytes_ += 2.0 * Hkv * d * e * P + (2.0 * Hq + 4.0 * Hkv) * d * e * Lq
+    return flops, bytes_
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        # keep samples taken under load (upper half) for the median
+        sm_sorted = sorted(sm)
+        load = sm_sorted[len(sm_sorted) // 2:] if sm_sorted else []
+        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# oracle timing (cpu_baseline leg and the --impl reference arm)
+# ---------------------------------------------------------------------------------------------------
+
+def oracle_sample(spec, wl, n_tokens: int = 0):
+    """Time the fp64 oracle, as it stands, on layer 0 of every request: composition + re-basing of the
+    whole prefix, then attention for every head of `n_tokens` query tokens (0 = all).  Returns the
+    job-level rate it implies: query tokens/s through the full stack = batch*q_len / (L * sum_b t_b)."""
+    from oracle import reference as orc
+    s = spec.shape
+    ad = wl.adapter_host()
+    f = orc.inv_freq(s.rope_theta, s.head_dim)
+    q, kn, vn = wl.query_layer(0)
+    # pull the bytes to the host before timing (the oracle's inputs are host arrays)
+    cached = {}
+    for it in spec.items:
+        for pid, _ in it:
+            if pid not in cached:
+                cached[pid] = wl.packet_layer(pid, 0)
+    st = orc.Store(s.dtype)
+    for pid, n in enumerate(spec.packet_lens):
+        st.register_packet(n, 0, (lambda layer, pid=pid: cached[pid]))
+    st.register_adapter(ad.n_header, 0, ad.n_trailer, 0, (lambda layer: (ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0])))
+    toks = list(range(spec.q_len))
+    if n_tokens > 0:
+        pick = sorted(set([0, 1, 63, 64, 127, 128, spec.q_len - 1]) & set(toks))
+        toks = pick[:n_tokens]
+    rows = [(h, i) for i in toks for h in range(s.n_q_heads)]
+    t_total = t_comp = t_att = 0.0
+    for b in range(spec.batch):
+        t0 = time.perf_counter()
+        plan = orc.compose(st, spec.items[b], spec.rebase)
+        Kp, Vp, _ = orc.composed_kv(st, plan, 0, f, s.rope_pairing)
+        t1 = time.perf_counter()
+        Q = orc.widen(q[b], s.dtype)
+        K = np.concatenate([Kp, orc.widen(kn[b], s.dtype)])
+        V = np.concatenate([Vp, orc.widen(vn[b], s.dtype)])
+        orc.attention_rows(K, V, Q, plan.prefix_len, 1.0 / np.sqrt(s.head_dim), rows)
+        t2 = time.perf_counter()
+        t_comp += t1 - t0
+        t_att += t2 - t1
+        t_total += (t1 - t0) + (t2 - t1) / len(rows) * (spec.q_len * s.n_q_heads)
+    tokens_per_s = spec.batch * spec.q_len / (s.n_layers * t_total)
+    return {"value": tokens_per_s, "unit": "tokens/s", "cores": orc.threads(), "kind": "oracle",
+            "sample": f"layer 0 of all {spec.batch} requests: compose + re-base of the prefix ({t_comp:.2f} s) and attention "
+                      f"rows of {len(toks)} of {spec.q_len} query tokens x {s.n_q_heads} heads ({t_att:.2f} s); scaled to "
+                      f"{spec.q_len} tokens x {s.n_layers} layers",
+            "seconds": t_comp + t_att}
+
+
+# ---------------------------------------------------------------------------------------------------
+# extra roofline points (memory-bound shape, gather kernel)
+# ---------------------------------------------------------------------------------------------------
+
+def flush_l2(torch, dev, buf=[None]):
+    if buf[0] is None:
+        buf[0] = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    buf[0].zero_()
+
+
+def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peaks, device: int):
+    """ms of one layer's attention kernel (CUDA events inside the library) and of the gather kernel."""
+    import torch
+    from paper_2604_13226_b200 import binding as kvp, inputs as gen
+    from paper_2604_13226_b200.session import Session
+    spec = make_spec(spec_name, seed)
+    wl = gen.DeviceWorkload(spec, f"cuda:{device}")
+    sess = Session(wl, materialize=materialize, device=device)
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 1)
+    dev = torch.device(f"cuda:{device}")
+    qkv = sess.query_tensors(0)
+    att, gat = [], []
+    for it in range(iters + 3):
+        flush_l2(torch, dev)
+        sess.assemble()
+        flush_l2(torch, dev)
+        sess.prefill(0, qkv=qkv, want_lse=False)
+        torch.cuda.synchronize(dev)
+        a, g = sess.ctx.kernel_times(0), sess.ctx.kernel_times(1)
+        if it >= 3:
+            att += a
+            gat += g
+    launch = sess.ctx.last_launch()
+    assert sess.ctx.status_word() == 0
+    flops, bytes_ = algorithmic_work(spec)
+    s = spec.shape
+    tok_bytes = 2.0 * s.n_kv_heads * s.head_dim * s.elem_bytes
+    if materialize:
+        moved = sum(spec.prefix_len(b) for b in range(spec.batch))
+    else:
+        moved = sum(spec.prefix_len(b) - sum(spec.packet_lens[p] for p, _ in spec.items[b]) for b in range(spec.batch))
+    gather_bytes = 2.0 * moved * tok_bytes * s.n_layers           # read + write, all layers
+    ms_a = statistics.median(att)
+    ms_g = statistics.median(gat) if gat else None
+    sess.close()
+    del sess, wl
+    torch.cuda.empty_cache()
+    res = {"workload": spec.name, "attn_ms": ms_a, "attn_tflops": flops / ms_a / 1e9, "attn_gbs": bytes_ / ms_a / 1e6,
+           "frac_tensor_sustained": flops / ms_a / 1e9 / peaks["bf16_tflops_sustained"],
+           "frac_hbm": bytes_ / ms_a / 1e6 / peaks["hbm_gbs"], "launch": launch, "l2": "flushed between iterations"}
+    if ms_g:
+        res.update({"gather_ms": ms_g, "gather_gbs": gather_bytes / ms_g / 1e6,
+                    "gather_frac_hbm": gather_bytes / ms_g / 1e6 / peaks["hbm_gbs"], "gather_bytes": gather_bytes})
+    return res
+
+
+# ---------------------------------------------------------------------------------------------------
+# main
+# ---------------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config3")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-extras", action="store_true", help="skip the extra roofline points and the CPU baseline")
+    ap.add_argument("--materialize", action="store_true", help="materialise the composed prefix instead of reading in place")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    peaks = load_peaks()
+
+    import torch
+    from paper_2604_13226_b200 import inputs as gen
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        spec = make_spec(args.workload, args.seed)
+        dev = "cuda:0" if torch.cuda.is_available() else None
+        if dev is None:
+            print(json.dumps({"impl": "reference", "unavailable": "the seeded workload generator needs a CUDA device"}))
+            return
+        wl = gen.DeviceWorkload(spec, dev)
+        for _ in range(args.warmup):
+            oracle_sample(spec, wl, n_tokens=1)
+        t0 = time.perf_counter()
+        vals = [oracle_sample(spec, wl, n_tokens=0 if args.steps <= 4 else 5) for _ in range(max(1, args.steps))]
+        dt = time.perf_counter() - t0
+        v = statistics.median(x["value"] for x in vals)
+        cb = dict(vals[-1])
+        cb["value"] = v
+        s = spec.shape
+        print(json.dumps({
+            "impl": "reference", "metric": "composed_cache_prefill_query_tokens_per_s", "value": v, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": spec.batch * spec.q_len / v * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": spec.name, "layers": s.n_layers, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
+                       "head_dim": s.head_dim, "batch": spec.batch, "q_len": spec.q_len,
+                       "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)],
+                       "note": "each step = a bounded sample of the workload run through the CPU oracle"},
+            "cpu_baseline": cb, "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "wall_s": dt}))
+        return
+
+    # ---- our arm ---------------------------------------------------------------------------------
+    from paper_2604_13226_b200 import binding as kvp
+    from paper_2604_13226_b200.session import Session
+    kvp.lib()                                                    # fail loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device(f"cuda:{local_rank}")
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    spec = make_spec(args.workload, args.seed + 17 * rank)         # weak scaling: every rank its own batch
+    s = spec.shape
+    wl = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
+    sess = Session(wl, materialize=args.materialize, device=local_rank)
+    L = s.n_layers
+    qkv = [sess.query_tensors(l) for l in range(L)]
+    outs = [torch.empty_like(qkv[l][0]) for l in range(L)]
+    Lq = spec.q_len
+
+    def step():
+        sess.assemble()
+        for l in range(L):
+            q, kn, vn = qkv[l]
+            sess.ctx.query_prefill(sess.assembly_id, l, q, kn, vn, Lq, outs[l], None, 0)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches_per_step = 1 + L * sess.ctx.last_launch()["launches"]
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 1)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev0.elapsed_time(ev1)
+    attn_ms = sess.ctx.kernel_times(0)
+    gather_ms = sess.ctx.kernel_times(1)
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 0)
+    status = sess.ctx.status_word()
+    assert status == 0, f"device status word {status}"
+    launch = sess.ctx.last_launch()
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ------------
+    hq = [tuple(t.cpu().pin_memory() for t in qkv[l]) for l in range(L)]
+    hout = [torch.empty_like(outs[l], device="cpu").pin_memory() for l in range(L)]
+    dq = tuple(torch.empty_like(t) for t in qkv[0])
+    dout = torch.empty_like(outs[0])
+    h2d = sum(t.numel() * t.element_size() for t in hq[0]) * L
+    d2h = hout[0].numel() * hout[0].element_size() * L
+
+    def step_e2e():
+        sess.assemble()
+        for l in range(L):
+            for dst, src in zip(dq, hq[l]):
+                dst.copy_(src, non_blocking=True)
+            sess.ctx.query_prefill(sess.assembly_id, l, dq[0], dq[1], dq[2], Lq, dout, None, 0)
+            hout[l].copy_(dout, non_blocking=True)
+
+    for _ in range(3):
+        step_e2e()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+
+    sess.close()
+    del sess
+    torch.cuda.empty_cache()
+
+    if rank == 0:
+        tokens = spec.batch * Lq * world
+        ms_step = ms_total / args.steps
+        value = tokens / (ms_step * 1e-3)
+        flops, bytes_ = algorithmic_work(spec)
+        a_ms = statistics.mean(attn_ms) if attn_ms else None
+        tensor_bound = s.group * Lq >= 247
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+        if os.path.exists(tpath):
+            traffic = json.load(open(tpath)).get(spec.name)
+        if a_ms:
+            if tensor_bound:
+                ach = flops / a_ms / 1e9
+                roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                        "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
+                        "peak_source": peaks["source"] + " (sustained bf16 GEMM; burst %.1f)" % peaks["bf16_tflops"]}
+            else:
+                ach = bytes_ / a_ms / 1e6
+                roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": peaks["source"]}
+            roof.update({"kernel": "attn_sm100_kernel", "launches_timed": len(attn_ms), "avg_launch_ms": a_ms,
+                         "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
+                         "attn_share_of_step": sum(attn_ms) / ms_total,
+                         "gather_avg_ms": statistics.mean(gather_ms) if gather_ms else None})
+        else:
+            roof = None
+        line = {
+            "metric": "composed_cache_prefill_query_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": spec.name, "layers": L, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
+                       "head_dim": s.head_dim, "batch_per_gpu": spec.batch, "q_len": Lq,
+                       "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)], "rope_theta": s.rope_theta,
+                       "mode": "materialised cache" if args.materialize else "fused in place (adapters staged)",
+                       "l2": "inputs larger than L2: every layer reads %.0f MB of distinct K/V" % (bytes_ / 1e6),
+                       "sharding": "requests sharded across ranks, no collective"},
+            "prefix_tokens_per_s": sum(spec.prefix_len(b) for b in range(spec.batch)) * world / (ms_step * 1e-3),
+            "e2e": {"value": tokens / (ms_e2e / args.steps * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e / args.steps,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * args.steps, "launch": launch, "roofline": roof, "clocks": clocks,
+        }
+        if not args.no_extras and world == 1:
+            extras = {}
+            try:
+                extras["hbm_bound_point"] = measure_point("config5:64:16:1", args.seed, 10, False, peaks, local_rank)
+                extras["gather_materialise_point"] = measure_point("config5:16:64:1", args.seed, 10, True, peaks, local_rank)
+            except Exception as ex:                                   # extras never invalidate the main line
+                extras["error"] = repr(ex)
+            line["extra_points"] = extras
+            wl2 = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
+            line["cpu_baseline"] = oracle_sample(spec, wl2)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

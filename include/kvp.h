@@ -192,9 +192,17 @@ KVP_API int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int3
 
 /* Launch tuning (not needed for correctness).  key KVP_TUNE_SPLIT_TARGET_CTAS: the tcgen05 path
    splits each request's keys until about `value` CTAs exist (0 = default, 4 per SM);
-   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic). */
-enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2 };
+   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic);
+   key KVP_TUNE_TIME_KERNELS: value != 0 brackets every attention and gather kernel with CUDA events
+   on the caller's stream (up to 4096 launches between two kvp_kernel_times calls). */
+enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3 };
 KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);
+
+/* Device durations, in milliseconds, of the kernels launched since the last call with this `which`
+   (0 = main attention kernel of kvp_query_prefill, 1 = gather kernel of kvp_assemble), oldest first;
+   needs KVP_TUNE_TIME_KERNELS.  Synchronises on the recorded events.  ms: host array of `cap`
+   floats; *n receives the number written. */
+KVP_API int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t cap, int32_t *n);
 
 /* Text of the last error on this context (owned by ctx; "" if none).  With ctx == NULL: the reason
    the last kvp_create on this thread failed. */

@@ -19,7 +19,7 @@ STATUS_NAMES = {0: "KVP_OK", 1: "KVP_ERR_INVALID", 2: "KVP_ERR_CAPACITY", 3: "KV
 DTYPE_F32, DTYPE_BF16 = 0, 1
 REBASE, MATERIALIZE = 1, 2
 ROPE_QUERY, FORCE_SIMPLE = 1, 2
-TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS = 1, 2
+TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS = 1, 2, 3
 
 
 class KvpError(RuntimeError):
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         "kvp_status_word": (i32, [vp, pi32]),
         "kvp_last_launch": (i32, [vp, pi32, pi32, pi32, pi32]),
         "kvp_tune": (i32, [vp, i32, i32]),
+        "kvp_kernel_times": (i32, [vp, i32, ctypes.POINTER(ctypes.c_float), i32, pi32]),
         "kvp_last_error": (ctypes.c_char_p, [vp]),
     }
     for name, (res, args) in sig.items():
@@ -84,7 +85,7 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
             "kvp_export_plan", "kvp_export_cache", "kvp_status_word", "kvp_last_launch", "kvp_tune",
-            "kvp_last_error"]
+            "kvp_kernel_times", "kvp_last_error"]
 
 
 def _i32_array(xs: Sequence[int]):
@@ -253,3 +254,10 @@ class Context:
 
     def tune(self, key: int, value: int):
         self._check(self._L.kvp_tune(self._h, key, value))
+
+    def kernel_times(self, which: int = 0, cap: int = 4096) -> List[float]:
+        """Device durations (ms) of the attention (0) / gather (1) kernels since the last call."""
+        buf = (ctypes.c_float * cap)()
+        n = ctypes.c_int32(0)
+        self._check(self._L.kvp_kernel_times(self._h, which, buf, cap, ctypes.byref(n)))
+        return [float(buf[i]) for i in range(n.value)]

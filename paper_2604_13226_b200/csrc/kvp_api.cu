@@ -113,6 +113,25 @@ bool make_tensor_map(encode_tiled_fn enc, CUtensorMap *tm, void *base, int head_
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr int kMaxTimed = 4096;
+
+// Record an event before (edge 0) / after (edge 1) a timed kernel; events are created on first use.
+cudaError_t time_edge(kvp_ctx *ctx, int which, int edge, cudaStream_t st)
+{
+    if (!ctx->time_kernels || ctx->tev_n[which] >= kMaxTimed) return cudaSuccess;
+    std::vector<cudaEvent_t> &v = ctx->tev[which][edge];
+    const int i = ctx->tev_n[which];
+    if ((int)v.size() <= i) {
+        cudaEvent_t e;
+        cudaError_t rc = cudaEventCreate(&e);
+        if (rc != cudaSuccess) return rc;
+        v.push_back(e);
+    }
+    cudaError_t rc = cudaEventRecord(v[i], st);
+    if (rc == cudaSuccess && edge == 1) ++ctx->tev_n[which];
+    return rc;
+}
+
 kvp_plan_dev plan_dev(const kvp_ctx *ctx, int slot)
 {
     char *base = ctx->slot_plan_dev[slot];
@@ -265,6 +284,7 @@ int32_t kvp_destroy(kvp_ctx *ctx)
         cudaDeviceSynchronize();
         for (char *h : ctx->slot_plan_host) cudaFreeHost(h);
         for (cudaEvent_t e : ctx->slot_event) cudaEventDestroy(e);
+        for (auto &w : ctx->tev) for (auto &v : w) for (cudaEvent_t e : v) cudaEventDestroy(e);
     }
     delete ctx;
     return KVP_OK;
@@ -457,8 +477,10 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
         const uint64_t used = ctx->pl.rope + sizeof(float2) * rope_delta.size() * half;
         KVP_CUDA(ctx, cudaMemcpyAsync(ctx->slot_plan_dev[slot], h, used, cudaMemcpyHostToDevice, st));
         KVP_CUDA(ctx, cudaEventRecord(ctx->slot_event[slot], st));
+        KVP_CUDA(ctx, time_edge(ctx, 1, 0, st));
         KVP_CUDA(ctx, kvp_launch_gather(ctx->shape, plan_dev(ctx, slot), as.n_chunks, ctx->pool_k, ctx->pool_v,
                                         ctx->slot_k[slot], ctx->slot_v[slot], st));
+        KVP_CUDA(ctx, time_edge(ctx, 1, 1, st));
     }
     ctx->slots[slot] = std::move(as);
     *assembly_id = id;
@@ -536,8 +558,10 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
     int32_t ctas = 0, splits = 1;
     if (!fast) {
+        KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
         KVP_CUDA(ctx, kvp_launch_attn_simple(sh, plan, as.batch, q_len, layer, q_used, ctx->pool_k, ctx->pool_v,
                                              ctx->slot_k[slot], ctx->slot_v[slot], out, lse, &ctas, st));
+        KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
         ctx->last_kind = 0;
     } else {
@@ -566,8 +590,10 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         a.partial_o = ctx->partial_o;
         a.partial_ml = ctx->partial_ml;
         a.status = ctx->status_dev;
+        KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
         KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot],
                                             ctx->tm_ws_v[slot], &ctas, st));
+        KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
         if (splits > 1) {
             KVP_CUDA(ctx, kvp_launch_merge(sh, as.batch, q_len, splits, n_mtiles, ctx->partial_o, ctx->partial_ml, out,
@@ -606,11 +632,26 @@ int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int32_t *spl
     return KVP_OK;
 }
 
+int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t cap, int32_t *n)
+{
+    if (!ctx || !n || which < 0 || which > 1 || (cap > 0 && !ms)) return KVP_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "kernel_times: host-only context");
+    const int cnt = std::min(cap, ctx->tev_n[which]);
+    for (int i = 0; i < cnt; ++i) {
+        KVP_CUDA(ctx, cudaEventSynchronize(ctx->tev[which][1][i]));
+        KVP_CUDA(ctx, cudaEventElapsedTime(&ms[i], ctx->tev[which][0][i], ctx->tev[which][1][i]));
+    }
+    *n = cnt;
+    ctx->tev_n[which] = 0;
+    return KVP_OK;
+}
+
 int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
 {
     if (!ctx) return KVP_ERR_INVALID;
     if (key == KVP_TUNE_SPLIT_TARGET_CTAS) ctx->split_target_ctas = value;
     else if (key == KVP_TUNE_FORCE_SPLITS) ctx->force_splits = value;
+    else if (key == KVP_TUNE_TIME_KERNELS) { ctx->time_kernels = value != 0; ctx->tev_n[0] = ctx->tev_n[1] = 0; }
     else return fail(ctx, KVP_ERR_INVALID, "tune: unknown key %d", key);
     return KVP_OK;
 }
