@@ -204,6 +204,41 @@ KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);
    floats; *n receives the number written. */
 KVP_API int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t cap, int32_t *n);
 
+/*
+ * Gather + re-base of one request's segments with NO allocation anywhere (the paper has no
+ * counterpart of this call; it exists for integration).  It is the gather kernel of kvp_assemble
+ * for callers that cannot provide a workspace and must not trigger any allocation: code that runs
+ * after the process's device heap has been frozen, plugins that receive raw device pointers but no
+ * allocator, callbacks that may not enter the CUDA allocator.  It needs no kvp_ctx.
+ *
+ * Segment s (pool rows [src_row0[s], src_row0[s] + seg_len[s]) of every plane) is copied behind
+ * segment s-1 into the cache, starting at cache row 0; its keys are rotated by delta[s] positions
+ * (Eq. 1; theta_i = rope_theta^(-2i/d); angles in double precision on the device), its values are
+ * byte copies.  A plane is one (layer, kv head): pool_k/pool_v are [n_planes][pool_rows][head_dim],
+ * cache_k/cache_v are [n_planes][cache_rows][head_dim], all device pointers the caller owns, 16-byte
+ * aligned.  src_row0, seg_len, delta are host arrays, read before the call returns.
+ *
+ * Scratch: the per-segment records and cos/sin tables live in a fixed array inside the library image,
+ * 50,688 bytes on every GPU that loads the library, sized for KVP_NOALLOC_MAX_SEGMENTS segments per
+ * call; more segments are refused with KVP_ERR_CAPACITY (split the request into several calls with
+ * cache pointers advanced by the rows already written).  The array is shared by all calls on a device
+ * and keeps the previous call's contents; every record a call reads is rewritten by that call first,
+ * so nothing depends on its old contents, but calls whose kernels can overlap on the GPU (different
+ * streams or threads) race on it and must be serialised by the caller.
+ *
+ * The first call on each device looks up the array's device address (the device must be current);
+ * make that first call outside any stream capture.  Two kernels are enqueued on `stream`; the call
+ * does not synchronise.  No cudaMalloc/cudaFree or other allocating routine is called.
+ * err (optional, err_cap bytes) receives a message on failure.
+ * Errors: INVALID (null pointer, bad shape/dtype, segment outside the pool), CAPACITY, CUDA.
+ */
+#define KVP_NOALLOC_MAX_SEGMENTS 96
+KVP_API int32_t kvp_compose_noalloc(const void *pool_k, const void *pool_v, int64_t pool_rows, int32_t n_planes,
+                                    int32_t head_dim, int32_t dtype, int32_t rope_pairing, double rope_theta,
+                                    int32_t n_segments, const int32_t *src_row0, const int32_t *seg_len,
+                                    const int32_t *delta, void *cache_k, void *cache_v, int64_t cache_rows,
+                                    void *stream, char *err, int32_t err_cap);
+
 /* Text of the last error on this context (owned by ctx; "" if none).  With ctx == NULL: the reason
    the last kvp_create on this thread failed. */
 KVP_API const char *kvp_last_error(kvp_ctx *ctx);

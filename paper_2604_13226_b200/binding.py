@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         "kvp_tune": (i32, [vp, i32, i32]),
         "kvp_kernel_times": (i32, [vp, i32, ctypes.POINTER(ctypes.c_float), i32, pi32]),
         "kvp_last_error": (ctypes.c_char_p, [vp]),
+        "kvp_compose_noalloc": (i32, [vp, vp, ctypes.c_int64, i32, i32, i32, i32, ctypes.c_double, i32, pi32, pi32, pi32,
+                                      vp, vp, ctypes.c_int64, vp, ctypes.c_char_p, i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)          # AttributeError if the library lacks a declared symbol
@@ -85,7 +87,7 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
             "kvp_export_plan", "kvp_export_cache", "kvp_status_word", "kvp_last_launch", "kvp_tune",
-            "kvp_kernel_times", "kvp_last_error"]
+            "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
 
 def _i32_array(xs: Sequence[int]):
@@ -261,3 +263,20 @@ class Context:
         n = ctypes.c_int32(0)
         self._check(self._L.kvp_kernel_times(self._h, which, buf, cap, ctypes.byref(n)))
         return [float(buf[i]) for i in range(n.value)]
+
+
+def compose_noalloc(pool_k: int, pool_v: int, pool_rows: int, n_planes: int, head_dim: int, dtype: str,
+                    rope_pairing: int, rope_theta: float, segments, cache_k, cache_v, cache_rows: int, stream=None):
+    """``kvp_compose_noalloc``: gather + re-base ``segments`` = [(src_row0, length, delta), ...] from the
+    caller's pool planes into the caller's cache planes without any allocation in the library.
+    ``pool_k``/``pool_v`` are device addresses, ``cache_k``/``cache_v`` torch tensors (or addresses)."""
+    L = lib()
+    n = len(segments)
+    err = ctypes.create_string_buffer(256)
+    st = ctypes.c_void_p(stream.cuda_stream) if stream is not None else None
+    rc = L.kvp_compose_noalloc(pool_k, pool_v, pool_rows, n_planes, head_dim, DTYPE_BF16 if dtype == "bf16" else DTYPE_F32,
+                               rope_pairing, rope_theta, n, _i32_array([s[0] for s in segments]),
+                               _i32_array([s[1] for s in segments]), _i32_array([s[2] for s in segments]),
+                               _ptr(cache_k), _ptr(cache_v), cache_rows, st, err, 256)
+    if rc != KVP_OK:
+        raise KvpError(rc, err.value.decode())
