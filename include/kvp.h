@@ -182,6 +182,23 @@ KVP_API int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t laye
                          int32_t n_query_rows, void *k_out, void *v_out, int32_t k_as_f32,
                          void *stream);
 
+/*
+ * The work list the tensor-core attention kernel would use for `q_len` query tokens over this assembly
+ * (host arrays, any may be NULL; works in a host-only context).  The kernel is persistent: CTA c runs
+ * pieces [cta_begin[c], cta_begin[c+1]).  A piece is 8 ints {request, kv head, first packed query row
+ * of its unit, mode, first key tile, number of key tiles, partial slot of stream 0, of stream 1};
+ * a unit is <= 256 packed rows (query token, head-in-group) of one request and kv head, its key tiles
+ * numbered with the causal tiles of the query's own keys first and the request's prefix tiles after
+ * them; mode 0 = two 128-row query tiles over every key tile, mode 1 = one query tile whose key tiles
+ * alternate between the CTA's two streams; slot -1 = the piece covers the unit's whole key range and
+ * writes the output directly.  A merge item is 8 ints {request, kv head, first packed row, first
+ * partial slot, number of slots, 0, 0, 0}.  counts (4 ints): CTAs, pieces, merge items, partial slots.
+ * Errors: NOT_FOUND, INVALID, CAPACITY (an output array is too small; counts is still written).
+ */
+KVP_API int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, int32_t *cta_begin,
+                                    int32_t cta_cap, int32_t *works, int32_t work_cap, int32_t *merges,
+                                    int32_t merge_cap, int32_t *counts);
+
 /* Synchronises the device and returns the device-side status word (0 = no bounded wait ran out;
    otherwise a code identifying the wait) in *device_status, then clears it. */
 KVP_API int32_t kvp_status_word(kvp_ctx *ctx, int32_t *device_status);
@@ -192,10 +209,12 @@ KVP_API int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int3
 
 /* Launch tuning (not needed for correctness).  key KVP_TUNE_SPLIT_TARGET_CTAS: the tcgen05 path
    splits each request's keys until about `value` CTAs exist (0 = default, 4 per SM);
-   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic);
+   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic; for the two-stream kernel only
+   1 is meaningful: no unit is split);
+   key KVP_TUNE_KERNEL_VARIANT: 0 = two-stream persistent tcgen05 kernel (default), 1 = single-tile kernel;
    key KVP_TUNE_TIME_KERNELS: value != 0 brackets every attention and gather kernel with CUDA events
    on the caller's stream (up to 4096 launches between two kvp_kernel_times calls). */
-enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3 };
+enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3, KVP_TUNE_KERNEL_VARIANT = 4 };
 KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);
 
 /* Device durations, in milliseconds, of the kernels launched since the last call with this `which`

@@ -19,7 +19,7 @@ STATUS_NAMES = {0: "KVP_OK", 1: "KVP_ERR_INVALID", 2: "KVP_ERR_CAPACITY", 3: "KV
 DTYPE_F32, DTYPE_BF16 = 0, 1
 REBASE, MATERIALIZE = 1, 2
 ROPE_QUERY, FORCE_SIMPLE = 1, 2
-TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS = 1, 2, 3
+TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS, TUNE_KERNEL_VARIANT = 1, 2, 3, 4
 
 
 class KvpError(RuntimeError):
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
         "kvp_export_plan": (i32, [vp, i32, i32, pi32, pi32, pi32, pi32]),
         "kvp_export_cache": (i32, [vp, i32, i32, i32, i32, vp, vp, i32, vp]),
+        "kvp_export_schedule": (i32, [vp, i32, i32, pi32, i32, pi32, i32, pi32, i32, pi32]),
         "kvp_status_word": (i32, [vp, pi32]),
         "kvp_last_launch": (i32, [vp, pi32, pi32, pi32, pi32]),
         "kvp_tune": (i32, [vp, i32, i32]),
@@ -86,7 +87,7 @@ def lib() -> ctypes.CDLL:
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
-            "kvp_export_plan", "kvp_export_cache", "kvp_status_word", "kvp_last_launch", "kvp_tune",
+            "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
 
@@ -241,6 +242,20 @@ class Context:
         self._check(self._L.kvp_export_cache(self._h, assembly_id, layer, b, n_query_rows, _ptr(k), _ptr(v),
                                              1 if k_as_f32 else 0, self._stream(stream)))
         return k, v
+
+    def export_schedule(self, assembly_id: int, q_len: int):
+        """(cta_begin [n_ctas+1], works [n][8], merges [m][8], n_slots) as numpy int32 arrays."""
+        import numpy as np
+        pi = ctypes.POINTER(ctypes.c_int32)
+        counts = (ctypes.c_int32 * 4)()
+        self._check(self._L.kvp_export_schedule(self._h, assembly_id, q_len, None, 0, None, 0, None, 0, counts))
+        cb = np.zeros(counts[0] + 1, dtype=np.int32)
+        works = np.zeros((max(1, counts[1]), 8), dtype=np.int32)
+        merges = np.zeros((max(1, counts[2]), 8), dtype=np.int32)
+        self._check(self._L.kvp_export_schedule(self._h, assembly_id, q_len, cb.ctypes.data_as(pi), cb.size,
+                                                works.ctypes.data_as(pi), works.shape[0],
+                                                merges.ctypes.data_as(pi), merges.shape[0], counts))
+        return cb, works[:counts[1]], merges[:counts[2]], int(counts[3])
 
     def status_word(self) -> int:
         w = ctypes.c_int32(0)

@@ -20,9 +20,31 @@ constexpr uint64_t kAlign = 1024;
 inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 struct ws_layout {
-    uint64_t status, inv_freq, slots, slot_stride, slot_plan, slot_k, slot_v, partial_o, partial_ml, q_scratch, total;
+    uint64_t status, inv_freq, slots, slot_stride, slot_plan, slot_sched, slot_k, slot_v, partial_o, partial_ml, q_scratch, total;
     uint64_t rows_bytes;
 };
+
+constexpr int kMaxCtas = 256;          // upper bound on persistent CTAs (one per SM)
+
+// Work list of the two-stream attention kernel: [cta_begin: kMaxCtas + 1 ints][works][merge items].
+struct sched_layout {
+    uint64_t works, merges, total;
+    int32_t max_works, max_merges;
+};
+
+sched_layout schedule_layout(const kvp_config *c)
+{
+    sched_layout s;
+    const int group = c->n_q_heads / c->n_kv_heads;
+    const int64_t tiles_q = ((int64_t)group * c->max_query_tokens + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
+    const int64_t units = (int64_t)c->max_batch * c->n_kv_heads * tiles_q;
+    s.max_works = (int32_t)std::min<int64_t>(units + kMaxCtas, 1 << 24);
+    s.max_merges = 2 * kMaxCtas + 8;
+    s.works = round_up(4 * (kMaxCtas + 1), 256);
+    s.merges = round_up(s.works + sizeof(kvp_work) * (uint64_t)s.max_works, 256);
+    s.total = round_up(s.merges + sizeof(kvp_merge_item) * (uint64_t)s.max_merges, 256);
+    return s;
+}
 
 bool valid_cfg(const kvp_config *c)
 {
@@ -67,7 +89,8 @@ ws_layout workspace_layout(const kvp_config *c)
     w.inv_freq = o; o = round_up(o + 8 * 64, kAlign);
     w.rows_bytes = round_up((uint64_t)c->n_layers * c->n_kv_heads * c->max_ws_rows * c->head_dim * e, kAlign);
     w.slot_plan = 0;
-    w.slot_k = round_up(p.total, kAlign);
+    w.slot_sched = round_up(p.total, kAlign);
+    w.slot_k = round_up(w.slot_sched + schedule_layout(c).total, kAlign);
     w.slot_v = w.slot_k + w.rows_bytes;
     w.slot_stride = w.slot_v + w.rows_bytes;
     w.slots = o;    o += w.slot_stride * c->max_assemblies;
@@ -151,6 +174,155 @@ int find_slot(kvp_ctx *ctx, int32_t assembly_id)
     return ctx->slots[slot].id == assembly_id ? slot : -1;
 }
 
+// Work list of the two-stream kernel for one assembly and query length.  Units (<= 256 packed query
+// rows of one request and kv head) are laid end to end, each weighted by the tensor-core work of its
+// key tiles, and the line is cut into equal shares, one per CTA; a cut closer than two tiles to a unit
+// boundary moves onto it.  A unit that ends up in several pieces gets partial slots and merge items.
+struct schedule_t {
+    std::vector<int32_t> cta_begin;
+    std::vector<kvp_work> works;
+    std::vector<kvp_merge_item> merges;
+    int32_t n_ctas = 0, n_slots = 0, max_pieces = 1;
+};
+
+int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, schedule_t &out)
+{
+    const kvp_shape &sh = ctx->shape;
+    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces; };
+    std::vector<unit_t> units;
+    const int n_rows = sh.group * q_len;
+    int64_t total = 0;
+    for (int b = 0; b < as.batch; ++b) {
+        const int n_prefix = as.items[b].tile_end - as.items[b].tile_begin;
+        for (int hk = 0; hk < sh.n_kv_heads; ++hk)
+            for (int row_base = 0; row_base < n_rows; row_base += 2 * KVP_TILE_ROWS) {
+                unit_t u;
+                u.b = b; u.hk = hk; u.row_base = row_base;
+                u.mode = (n_rows - row_base <= KVP_TILE_ROWS) ? 1 : 0;
+                const int last = std::min(n_rows - 1, row_base + (u.mode ? 1 : 2) * KVP_TILE_ROWS - 1);
+                u.n_all = (last / sh.group) / KVP_TILE_KEYS + 1 + n_prefix;
+                u.first_piece = u.n_pieces = 0;
+                units.push_back(u);
+                total += (int64_t)u.n_all * (u.mode ? 1 : 2);
+            }
+    }
+    int G = std::min(ctx->sm_count, kMaxCtas);
+    if (ctx->split_target_ctas > 0) G = std::min(ctx->split_target_ctas, kMaxCtas);
+    if (total / G < 8) G = (int)std::max<int64_t>(1, total / 8);
+    const bool no_split = ctx->force_splits == 1;               // cuts only between units
+
+    // cut positions (unit, tile), non-decreasing
+    struct cut_t { int32_t u, t; };
+    std::vector<cut_t> cuts;
+    cuts.push_back({0, 0});
+    {
+        size_t u = 0;
+        int64_t c_u = 0;                                        // cost before unit u
+        for (int c = 1; c < G; ++c) {
+            const int64_t target = total * c / G;
+            while (u < units.size()) {
+                const int64_t cu = (int64_t)units[u].n_all * (units[u].mode ? 1 : 2);
+                if (target < c_u + cu) break;
+                c_u += cu;
+                ++u;
+            }
+            if (u >= units.size()) break;
+            const int w = units[u].mode ? 1 : 2;
+            int32_t t = (int32_t)((target - c_u + w / 2) / w);
+            if (no_split) t = (2 * t >= units[u].n_all) ? units[u].n_all : 0;
+            if (t < 2) t = 0;
+            if (units[u].n_all - t < 2) { cuts.push_back({(int32_t)u + 1, 0}); continue; }
+            cuts.push_back({(int32_t)u, t});
+        }
+    }
+    cuts.push_back({(int32_t)units.size(), 0});
+
+    std::vector<kvp_work> &works = out.works;
+    std::vector<int32_t> &cta_begin = out.cta_begin;
+    for (size_t c = 0; c + 1 < cuts.size(); ++c) {
+        const cut_t a = cuts[c], z = cuts[c + 1];
+        const size_t before = works.size();
+        for (int32_t u = a.u; u <= z.u && u < (int32_t)units.size(); ++u) {
+            const int32_t lo = (u == a.u) ? a.t : 0;
+            const int32_t hi = (u == z.u) ? z.t : units[u].n_all;
+            if (hi <= lo) continue;
+            kvp_work w;
+            w.b = units[u].b; w.hk = units[u].hk; w.row_base = units[u].row_base; w.mode = units[u].mode;
+            w.tile_lo = lo; w.n_tiles = hi - lo; w.slot0 = w.slot1 = -1;
+            if (units[u].n_pieces == 0) units[u].first_piece = (int32_t)works.size();
+            ++units[u].n_pieces;
+            works.push_back(w);
+        }
+        if (works.size() > before) cta_begin.push_back((int32_t)before);
+    }
+    const int n_ctas = (int)cta_begin.size();
+    cta_begin.push_back((int32_t)works.size());
+
+    std::vector<kvp_merge_item> &merges = out.merges;
+    int32_t n_slots = 0, max_pieces = 1;
+    for (const unit_t &u : units) {
+        if (u.n_pieces <= 1) continue;
+        max_pieces = std::max(max_pieces, u.n_pieces);
+        const int32_t base = n_slots;
+        for (int i = 0; i < u.n_pieces; ++i) {
+            kvp_work &w = works[u.first_piece + i];      // the pieces of a unit are consecutive
+            w.slot0 = base + i;
+            if (u.mode == 0) w.slot1 = base + u.n_pieces + i;
+        }
+        kvp_merge_item m;
+        memset(&m, 0, sizeof m);
+        m.b = u.b; m.hk = u.hk; m.row_base = u.row_base; m.slot0 = base; m.n_slots = u.n_pieces;
+        merges.push_back(m);
+        n_slots += u.n_pieces;
+        if (u.mode == 0) {
+            m.row_base = u.row_base + KVP_TILE_ROWS;
+            m.slot0 = base + u.n_pieces;
+            merges.push_back(m);
+            n_slots += u.n_pieces;
+        }
+    }
+    if (n_ctas > kMaxCtas || (int)works.size() > ctx->sched_max_works || (int)merges.size() > ctx->sched_max_merges ||
+        n_slots > KVP_MAX_SPLIT_UNITS)
+        return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: work list overflow (%d ctas, %zu pieces, %zu merges, %d slots)",
+                    n_ctas, works.size(), merges.size(), n_slots);
+
+    out.n_ctas = n_ctas;
+    out.n_slots = n_slots;
+    out.max_pieces = max_pieces;
+    return KVP_OK;
+}
+
+int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len, cudaStream_t st)
+{
+    schedule_t sc;
+    const int32_t rc = plan_schedule(ctx, as, q_len, sc);
+    if (rc != KVP_OK) return rc;
+    const std::vector<int32_t> &cta_begin = sc.cta_begin;
+    const std::vector<kvp_work> &works = sc.works;
+    const std::vector<kvp_merge_item> &merges = sc.merges;
+    const int n_ctas = sc.n_ctas;
+    const int32_t max_pieces = sc.max_pieces;
+    KVP_CUDA(ctx, cudaEventSynchronize(ctx->sched_event[slot]));          // staging buffer free again?
+    char *h = ctx->slot_sched_host[slot];
+    memcpy(h, cta_begin.data(), 4 * cta_begin.size());
+    memcpy(h + ctx->sched_off_works, works.data(), sizeof(kvp_work) * works.size());
+    memcpy(h + ctx->sched_off_merges, merges.data(), sizeof(kvp_merge_item) * merges.size());
+    char *d = ctx->slot_sched_dev[slot];
+    KVP_CUDA(ctx, cudaMemcpyAsync(d, h, 4 * cta_begin.size(), cudaMemcpyHostToDevice, st));
+    KVP_CUDA(ctx, cudaMemcpyAsync(d + ctx->sched_off_works, h + ctx->sched_off_works, sizeof(kvp_work) * works.size(),
+                                  cudaMemcpyHostToDevice, st));
+    if (!merges.empty())
+        KVP_CUDA(ctx, cudaMemcpyAsync(d + ctx->sched_off_merges, h + ctx->sched_off_merges,
+                                      sizeof(kvp_merge_item) * merges.size(), cudaMemcpyHostToDevice, st));
+    KVP_CUDA(ctx, cudaEventRecord(ctx->sched_event[slot], st));
+    as.sched_q_len = q_len;
+    as.sched_ctas = n_ctas;
+    as.sched_works = (int32_t)works.size();
+    as.sched_merges = (int32_t)merges.size();
+    as.sched_slots = max_pieces;
+    return KVP_OK;
+}
+
 thread_local std::string g_create_error;
 
 }  // namespace
@@ -199,6 +371,14 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
         ctx->inv_freq[i] = cfg->inv_freq ? cfg->inv_freq[i] : pow(cfg->rope_theta, -2.0 * i / cfg->head_dim);
     ctx->cfg.inv_freq = nullptr;
     ctx->pl = plan_layout(cfg);
+    {
+        const sched_layout sl = schedule_layout(cfg);
+        ctx->sched_off_works = sl.works;
+        ctx->sched_off_merges = sl.merges;
+        ctx->sched_bytes = sl.total;
+        ctx->sched_max_works = sl.max_works;
+        ctx->sched_max_merges = sl.max_merges;
+    }
     ctx->slots.resize(cfg->max_assemblies);
     *out = ctx;
     if (ctx->host_only) {
@@ -230,6 +410,7 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
     for (int a = 0; a < cfg->max_assemblies; ++a) {
         char *s = ws + w.slots + w.slot_stride * a;
         ctx->slot_plan_dev.push_back(s + w.slot_plan);
+        ctx->slot_sched_dev.push_back(s + w.slot_sched);
         ctx->slot_k.push_back(s + w.slot_k);
         ctx->slot_v.push_back(s + w.slot_v);
     }
@@ -252,6 +433,13 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
             return bail(KVP_ERR_CUDA, "pinned staging allocation failed");
         ctx->slot_plan_host.push_back(h);
         ctx->slot_event.push_back(ev);
+        char *hs = nullptr;
+        cudaEvent_t evs;
+        if (cudaHostAlloc((void **)&hs, ctx->sched_bytes, cudaHostAllocDefault) != cudaSuccess ||
+            cudaEventCreateWithFlags(&evs, cudaEventDisableTiming) != cudaSuccess)
+            return bail(KVP_ERR_CUDA, "pinned staging allocation failed");
+        ctx->slot_sched_host.push_back(hs);
+        ctx->sched_event.push_back(evs);
     }
 
     if (sh.dtype == KVP_DTYPE_BF16 && sh.head_dim == 128 && prop.major == 10) {
@@ -269,7 +457,8 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
                 ok = make_tensor_map(enc, &ctx->tm_ws_k[a], ctx->slot_k[a], sh.head_dim, sh.ws_rows, planes) &&
                      make_tensor_map(enc, &ctx->tm_ws_v[a], ctx->slot_v[a], sh.head_dim, sh.ws_rows, planes);
             if (!ok) return bail(KVP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-            if (kvp_attn_sm100_prepare() != cudaSuccess) return bail(KVP_ERR_CUDA, "tcgen05 kernel attribute setup failed");
+            if (kvp_attn_sm100_prepare() != cudaSuccess || kvp_attn_sm100_single_prepare() != cudaSuccess)
+                return bail(KVP_ERR_CUDA, "tcgen05 kernel attribute setup failed");
             ctx->have_tma = true;
         }
     }
@@ -284,6 +473,8 @@ int32_t kvp_destroy(kvp_ctx *ctx)
         cudaDeviceSynchronize();
         for (char *h : ctx->slot_plan_host) cudaFreeHost(h);
         for (cudaEvent_t e : ctx->slot_event) cudaEventDestroy(e);
+        for (char *h : ctx->slot_sched_host) cudaFreeHost(h);
+        for (cudaEvent_t e : ctx->sched_event) cudaEventDestroy(e);
         for (auto &w : ctx->tev) for (auto &v : w) for (cudaEvent_t e : v) cudaEventDestroy(e);
     }
     delete ctx;
@@ -564,6 +755,38 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
         ctx->last_kind = 0;
+    } else if (ctx->kernel_variant == 0) {
+        if (as.sched_q_len != q_len || as.sched_ctas == 0) {
+            const int32_t rc = build_schedule(ctx, as, slot, q_len, st);
+            if (rc != KVP_OK) return rc;
+        }
+        const char *sd = ctx->slot_sched_dev[slot];
+        kvp_attn2_args a;
+        a.plan = plan;
+        a.q_len = q_len;
+        a.layer = layer;
+        a.n_ctas = as.sched_ctas;
+        a.cta_begin = reinterpret_cast<const int32_t *>(sd);
+        a.works = reinterpret_cast<const kvp_work *>(sd + ctx->sched_off_works);
+        a.q = q_used;
+        a.out = out;
+        a.lse = lse;
+        a.partial_o = ctx->partial_o;
+        a.partial_ml = ctx->partial_ml;
+        a.status = ctx->status_dev;
+        KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
+        KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot], ctx->tm_ws_v[slot], st));
+        KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
+        ++launches;
+        if (as.sched_merges > 0) {
+            KVP_CUDA(ctx, kvp_launch_merge_list(sh, q_len, as.sched_merges,
+                                                reinterpret_cast<const kvp_merge_item *>(sd + ctx->sched_off_merges),
+                                                ctx->partial_o, ctx->partial_ml, out, lse, st));
+            ++launches;
+        }
+        ctas = as.sched_ctas;
+        splits = as.sched_slots;
+        ctx->last_kind = 1;
     } else {
         const int n_mtiles = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
         const int units = as.batch * sh.n_kv_heads * n_mtiles;
@@ -591,7 +814,7 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         a.partial_ml = ctx->partial_ml;
         a.status = ctx->status_dev;
         KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
-        KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot],
+        KVP_CUDA(ctx, kvp_launch_attn_sm100_single(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot],
                                             ctx->tm_ws_v[slot], &ctas, st));
         KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
@@ -632,6 +855,28 @@ int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int32_t *spl
     return KVP_OK;
 }
 
+int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, int32_t *cta_begin, int32_t cta_cap,
+                            int32_t *works, int32_t work_cap, int32_t *merges, int32_t merge_cap, int32_t *counts)
+{
+    if (!ctx || !counts) return KVP_ERR_INVALID;
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_schedule: unknown assembly %d", assembly_id);
+    if (q_len <= 0 || q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_INVALID, "export_schedule: bad q_len");
+    schedule_t sc;
+    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], q_len, sc);
+    if (rc != KVP_OK) return rc;
+    counts[0] = sc.n_ctas;
+    counts[1] = (int32_t)sc.works.size();
+    counts[2] = (int32_t)sc.merges.size();
+    counts[3] = sc.n_slots;
+    if ((cta_begin && cta_cap < sc.n_ctas + 1) || (works && work_cap < counts[1]) || (merges && merge_cap < counts[2]))
+        return fail(ctx, KVP_ERR_CAPACITY, "export_schedule: output arrays too small");
+    if (cta_begin) memcpy(cta_begin, sc.cta_begin.data(), 4 * sc.cta_begin.size());
+    if (works) memcpy(works, sc.works.data(), sizeof(kvp_work) * sc.works.size());
+    if (merges) memcpy(merges, sc.merges.data(), sizeof(kvp_merge_item) * sc.merges.size());
+    return KVP_OK;
+}
+
 int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t cap, int32_t *n)
 {
     if (!ctx || !n || which < 0 || which > 1 || (cap > 0 && !ms)) return KVP_ERR_INVALID;
@@ -649,8 +894,14 @@ int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t cap, in
 int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
 {
     if (!ctx) return KVP_ERR_INVALID;
-    if (key == KVP_TUNE_SPLIT_TARGET_CTAS) ctx->split_target_ctas = value;
-    else if (key == KVP_TUNE_FORCE_SPLITS) ctx->force_splits = value;
+    if (key == KVP_TUNE_SPLIT_TARGET_CTAS || key == KVP_TUNE_FORCE_SPLITS) {
+        (key == KVP_TUNE_SPLIT_TARGET_CTAS ? ctx->split_target_ctas : ctx->force_splits) = value;
+        for (kvp_assembly_host &as : ctx->slots) as.sched_q_len = 0;      // work lists are rebuilt on next use
+    }
+    else if (key == KVP_TUNE_KERNEL_VARIANT) {
+        if (value != 0 && value != 1) return fail(ctx, KVP_ERR_INVALID, "tune: kernel variant %d", value);
+        ctx->kernel_variant = value;
+    }
     else if (key == KVP_TUNE_TIME_KERNELS) { ctx->time_kernels = value != 0; ctx->tev_n[0] = ctx->tev_n[1] = 0; }
     else return fail(ctx, KVP_ERR_INVALID, "tune: unknown key %d", key);
     return KVP_OK;

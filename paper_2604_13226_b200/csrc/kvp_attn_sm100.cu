@@ -1,47 +1,65 @@
-// bf16 composed-cache attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMA with TMEM accumulators.
+// bf16 composed-cache attention for sm_100a: TMA-staged K/V tiles, tcgen05 MMA with TMEM accumulators,
+// two query streams per CTA so that the tensor pipe works on one stream while the other is in softmax.
 //
-// One CTA owns 128 packed query rows (query token i, head-in-group) of one (request, kv head) and a
-// contiguous range of that request's key tiles: first the causal tiles of the query's own keys, then
-// the prefix tiles of the plan (staged adapter rows, then documents read in place from the pool).
+// A persistent CTA (one per SM) walks a host-built list of work pieces.  A piece is a contiguous range
+// of the key tiles of one unit (<= 256 packed query rows - query token i, head-in-group - of one
+// request and kv head).  Key tiles are numbered per unit: the causal tiles of the query's own keys
+// first, then the prefix tiles of the plan (staged adapter rows, then documents read in place from
+// the pool).  The two streams of a piece are
+//   mode 0: query rows [0,128) and [128,256) of the unit, both visiting every key tile of the range;
+//   mode 1: the same 128 query rows twice, stream s visiting tiles lo+s, lo+s+2, ...; the two partial
+//           results are combined inside the CTA at the end of the piece.
 //
-//   warps 0-3  softmax: one thread per query row.  S = Q K^T arrives in TMEM; the thread takes the row
-//              max, forms p = exp2((s - m) * scale*log2e), sums it in fp32, writes P as bf16 back into
-//              TMEM over S, and rescales O in TMEM when the running max moved by more than 2^8.
-//              They also produce the Q operand: documents keep the keys they were cached with, so
-//              instead of rotating every key by Delta (Eq. 1) the Q tile is counter-rotated by -Delta
-//              once per document, which leaves every score q.k unchanged.
-//   warp 4     TMA producer: K then V of each tile into a 4-stage ring (two 64-column boxes each,
-//              128-byte swizzle).
-//   warp 5     MMA issuer: QK^T (both operands K-major in shared memory) into one of two S buffers,
-//              P V (P from TMEM, V MN-major in shared memory) accumulating into O; owns TMEM.
+//   warps 0-3 / 4-7   softmax of stream 0 / 1: one thread per query row.  S = Q K^T arrives in TMEM;
+//                     the thread takes the row max, forms p = exp2((s - m) * scale*log2e), sums it in
+//                     fp32, writes P as bf16 back into TMEM over S, and rescales O in TMEM when the
+//                     running max moved by more than 2^8.  At the end of a piece it normalises O and
+//                     writes the output rows (or an fp32 partial when the unit's keys are split).
+//   warps 8-11        Q producer.  Documents keep the keys they were cached with: instead of rotating
+//                     every key by Delta (Eq. 1) the 128-row Q tile of a stream is counter-rotated by
+//                     -Delta once per document, which leaves every score q.k unchanged.
+//   warp 12           MMA issuer and TMEM owner.  Per stream and step: O += P V of the previous tile,
+//                     then S = Q K^T of the next one; the two streams alternate.
+//   warp 13           TMA producer: K and V tiles into a 5-stage ring (two 64-column boxes each,
+//                     128-byte swizzle), in the order the MMA warp consumes them.
 //
 // Every mbarrier wait is bounded: when it runs out the CTA records a code in the status word, drains
 // what it has in flight, frees TMEM and returns.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "kvp_internal.h"
 
 namespace {
 
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kTileBytes = KVP_TILE_KEYS * 128 * 2;      // 32 KB: 128 rows x 128 bf16
 constexpr int kHalfBytes = kTileBytes / 2;               // one 64-column box
-constexpr int kThreads = 192;
+constexpr int kThreads = 512;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+constexpr uint32_t kColS = 0, kColO = 256;               // + 128 * stream
 
-constexpr int kOffQ = 0;                                  // 2 x 32 KB rotated-Q buffers
+constexpr int kOffQ = 0;                                  // one 32 KB rotated-Q buffer per stream
 constexpr int kOffRing = 2 * kTileBytes;                  // kStages x 32 KB
 constexpr int kOffBar = kOffRing + kStages * kTileBytes;
-constexpr int kSmemBytes = kOffBar + 256 + 1024;          // + barrier block + alignment slack
+constexpr int kOffMl = kOffBar + 256;                     // float2[128]: stream 1's (max, sum) in mode 1
+constexpr int kSmemBytes = kOffMl + 1024 + 1024;          // + alignment slack
 
-enum BarIdx { kKvFull = 0, kKvEmpty = kStages, kQFull = 2 * kStages, kSFull = kQFull + 2, kPFull = kSFull + 2,
-              kPvDone = kPFull + 2, kDrain = kPvDone + 2, kNumBars = kDrain + 1 };
+constexpr int kRegsSoftmax = 192, kRegsProducer = 72, kRegsIssue = 56;
+static_assert(2 * kRegsSoftmax + kRegsProducer + kRegsIssue <= 512, "register file");
+
+enum BarIdx { kKvFull = 0, kKvEmpty = kStages, kQFull = 2 * kStages, kQFree = kQFull + 2, kSFull = kQFree + 2,
+              kPFull = kSFull + 2, kOFull = kPFull + 2, kOFree = kOFull + 2, kMlFull = kOFree + 2, kDrain = kMlFull + 1,
+              kNumBars = kDrain + 1 };
+static_assert(8 * kNumBars + 8 <= 256, "barrier block");
 
 struct Params {
     kvp_plan_dev plan;
-    int batch, q_len, layer, n_splits, n_mtiles, n_q, n_kv, group, pairing;
+    int q_len, layer, n_q, n_kv, group, pairing;
     float scale, scale_log2;
+    const int32_t *cta_begin;
+    const kvp_work *works;
     const __nv_bfloat16 *q;
     __nv_bfloat16 *out;
     float *lse;
@@ -87,7 +105,7 @@ __device__ __forceinline__ uint64_t global_ns()
 
 // Bounded wait.  Returns false when another role has aborted or after ~2 s (then the status word and
 // the CTA's abort flag are set).  `code` identifies the wait.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                             int32_t *status, int code)
 {
     const uint64_t t0 = global_ns();
@@ -151,7 +169,7 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint3
 #define KVP_W8(r, o) "r"(r[o]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
 
 // 32 TMEM lanes (this warp's) x 32 consecutive 32-bit columns -> 32 registers per thread
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r)
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -161,7 +179,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r)
 {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -170,7 +188,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         ::"r"(taddr), KVP_W8(r, 0), KVP_W8(r, 8), KVP_W8(r, 16), KVP_W8(r, 24)
         : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r)
 {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -185,12 +203,20 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
 //   K-major operand (Q, K): rows are 128-byte lines; the leading-dimension field is unused (1).
@@ -210,28 +236,68 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major)
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// ---- work pieces and tiles ---------------------------------------------------------------------------
+
+struct Work {
+    int b, hk, row_base, mode, lo, n, slot0, slot1;
+    int n_tail, tile_begin, tail_row0, plane;
+    int steps0, steps1;
+};
+
+__device__ __forceinline__ Work load_work(const Params &p, int wi)
+{
+    const int4 *w4 = reinterpret_cast<const int4 *>(p.works + wi);
+    const int4 a = __ldg(w4), c = __ldg(w4 + 1);
+    Work w;
+    w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w;
+    w.lo = c.x; w.n = c.y; w.slot0 = c.z; w.slot1 = c.w;
+    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + w.b);
+    const int4 ia = __ldg(i4), ib = __ldg(i4 + 1);          // prefix_len, tile_begin, tile_end, seg_begin | seg_end, tail_row0, ..
+    w.tile_begin = ia.y;
+    w.tail_row0 = ib.y;
+    const int n_rows = p.group * p.q_len;
+    const int last = min(n_rows - 1, w.row_base + (w.mode ? KVP_TILE_ROWS : 2 * KVP_TILE_ROWS) - 1);
+    w.n_tail = (last / p.group) / KVP_TILE_KEYS + 1;
+    w.plane = p.layer * p.n_kv + w.hk;
+    w.steps0 = w.mode ? (w.n + 1) >> 1 : w.n;
+    w.steps1 = w.mode ? w.n >> 1 : w.n;
+    return w;
+}
+
 struct Tile {
     int row0, n_keys, src, rope, qoff;
 };
 
-__device__ __forceinline__ Tile get_tile(const Params &p, const kvp_item &it, int n_tail, int idx)
+// tile j of the unit's numbering
+__device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
 {
     Tile t;
-    if (idx < n_tail) {
-        t.row0 = it.tail_row0 + idx * KVP_TILE_KEYS;
-        t.n_keys = min(KVP_TILE_KEYS, p.q_len - idx * KVP_TILE_KEYS);
+    if (j < w.n_tail) {
+        t.row0 = w.tail_row0 + j * KVP_TILE_KEYS;
+        t.n_keys = min(KVP_TILE_KEYS, p.q_len - j * KVP_TILE_KEYS);
         t.src = 1;
         t.rope = 0;
-        t.qoff = idx * KVP_TILE_KEYS;
+        t.qoff = j * KVP_TILE_KEYS;
     } else {
-        const kvp_tile g = p.plan.tiles[it.tile_begin + idx - n_tail];
-        t.row0 = g.row0;
-        t.n_keys = g.n_keys;
-        t.src = g.src;
-        t.rope = g.rope;
+        const int4 g = __ldg(reinterpret_cast<const int4 *>(p.plan.tiles + w.tile_begin + (j - w.n_tail)));
+        t.row0 = g.x;
+        t.n_keys = g.y & 0xFFFF;
+        t.src = g.y >> 16;
+        t.rope = g.z;
         t.qoff = -1;
     }
     return t;
+}
+// unit tile number of step k of stream s
+__device__ __forceinline__ int stream_tile(const Work &w, int s, int k) { return w.lo + (w.mode ? 2 * k + s : k); }
+
+// Position of a K (kv = 0) or V (kv = 1) tile, r-th of the piece, in the piece's load order.
+//   mode 0: K0 V0 K1 V1 ...        mode 1: K0 K1 V0 K2 V1 K3 V2 ... V(n-1)
+__device__ __forceinline__ int load_seq(int mode, int n, int r, int kv)
+{
+    if (mode == 0) return 2 * r + kv;
+    if (kv == 0) return r == 0 ? 0 : 2 * r - 1;
+    return r <= n - 2 ? 2 * r + 2 : 2 * n - 1;
 }
 
 // Write this thread's query row, counter-rotated by the offset of rope-table row `rope`, into a
@@ -251,7 +317,7 @@ __device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t
     }
     const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
     const float2 *cs = p.plan.rope + (size_t)rope * 64;
-#pragma unroll
+#pragma unroll 2
     for (int c = 0; c < 8; ++c) {
         union { uint4 u; __nv_bfloat16 e[8]; } lo, hi;
         lo.u = __ldg(src + c);
@@ -285,64 +351,438 @@ __device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t
     }
 }
 
+struct Cta {
+    char *smem;
+    uint32_t smem_base, bar0, tmem;
+    volatile uint32_t *abort_flag;
+    int item_begin, item_end;
+    __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * i; }
+};
+
+// ---- softmax / correction / epilogue of stream S -------------------------------------------------------
+template <int S>
+__device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, const int t)
+{
+    const uint32_t lane_base = (uint32_t)((t >> 5) * 32) << 16;
+    const uint32_t s_addr = c.tmem + lane_base + kColS + S * 128;
+    const uint32_t o_addr = c.tmem + lane_base + kColO + S * 128;
+    const float c2 = p.scale_log2;
+    float2 *ml_smem = reinterpret_cast<float2 *>(c.smem + kOffMl);
+    uint32_t nS = 0, nO = 0, nMl = 0;
+    bool ok = true;
+
+    for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
+        const Work w = load_work(p, wi);
+        const int steps = S == 0 ? w.steps0 : w.steps1;
+        if (steps == 0) continue;
+        const int n_rows = p.group * p.q_len;
+        const int r = w.row_base + (w.mode == 0 ? S * KVP_TILE_ROWS : 0) + t;
+        const bool valid = r < n_rows;
+        const int qi = valid ? r / p.group : p.q_len - 1;
+        const int h = w.hk * p.group + (valid ? r % p.group : 0);
+
+        float m_ref = -1e30f, l = 0.f;
+        Tile nxt = get_tile(p, w, stream_tile(w, S, 0));
+        for (int k = 0; k < steps; ++k) {
+            const Tile tl = nxt;
+            if (k + 1 < steps) nxt = get_tile(p, w, stream_tile(w, S, k + 1));
+            ok = mbar_wait(c.bar(kSFull + S), nS & 1, c.abort_flag, p.status, 30 + S);
+            ++nS;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+
+            uint32_t v[128];
+            tmem_ld32(s_addr, v);
+            tmem_ld32(s_addr + 32, v + 32);
+            tmem_ld32(s_addr + 64, v + 64);
+            tmem_ld32(s_addr + 96, v + 96);
+            tc_wait_ld();
+
+            const bool full = (tl.n_keys == KVP_TILE_KEYS) && (tl.qoff < 0);
+            if (!full) {
+                const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);   // visible keys: [0, lim)
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (i >= lim) v[i] = 0xff800000u;                                          // -inf
+            }
+            float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]), mx2 = __uint_as_float(v[2]),
+                  mx3 = __uint_as_float(v[3]);
+#pragma unroll
+            for (int i = 4; i < 124; i += 8) {
+                mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                mx2 = fmax3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                mx3 = fmax3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+            }
+            mx0 = fmax3(mx0, __uint_as_float(v[124]), __uint_as_float(v[125]));
+            mx1 = fmax3(mx1, __uint_as_float(v[126]), __uint_as_float(v[127]));
+            const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
+            if (k == 0) {
+                m_ref = m_new;
+            } else {
+                const bool need = (m_new - m_ref) * c2 > 8.0f;
+                if (__any_sync(0xffffffffu, need)) {
+                    // S of this step is complete, hence so is the P V product of the previous step: O is quiet.
+                    const float alpha = need ? ex2((m_ref - m_new) * c2) : 1.f;
+                    if (need) m_ref = m_new;
+                    l *= alpha;
+#pragma unroll 1
+                    for (int ch = 0; ch < 8; ++ch) {
+                        uint32_t o[16];
+                        asm volatile(
+                            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                            : KVP_R8(o, 0), KVP_R8(o, 8)
+                            : "r"(o_addr + ch * 16)
+                            : "memory");
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st16(o_addr + ch * 16, o);
+                    }
+                }
+            }
+            // p = exp2((s - m) c), written over S as packed bf16 (columns 0..63 of the S block)
+            const float mc = m_ref * c2;
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                    const float p0 = ex2(fmaf(__uint_as_float(v[ch * 32 + i]), c2, -mc));
+                    const float p1 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 1]), c2, -mc));
+                    const float p2 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 2]), c2, -mc));
+                    const float p3 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 3]), c2, -mc));
+                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                    pk[i >> 1] = pack_bf16(p0, p1);
+                    pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+                }
+                tmem_st16(s_addr + ch * 16, pk);
+            }
+            l += (l0 + l1) + (l2 + l3);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(c.bar(kPFull + S));
+        }
+        if (!ok) break;
+
+        // ---- end of the piece: O of this stream is complete once its last P V has landed ----------
+        ok = mbar_wait(c.bar(kOFull + S), nO & 1, c.abort_flag, p.status, 32 + S);
+        ++nO;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+
+        if (w.mode == 1 && S == 1) {
+            ml_smem[t] = make_float2(m_ref, l);
+            mbar_arrive(c.bar(kMlFull));         // stream 0's warpgroup combines and writes
+            continue;
+        }
+        float w0 = 1.f, w1 = 0.f;
+        const bool both = (w.mode == 1) && (w.steps1 > 0);
+        if (both) {
+            ok = mbar_wait(c.bar(kMlFull), nMl & 1, c.abort_flag, p.status, 34);
+            ++nMl;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const float2 o = ml_smem[t];
+            const float M = fmaxf(m_ref, o.x);
+            w0 = ex2((m_ref - M) * c2);
+            w1 = ex2((o.x - M) * c2);
+            l = w0 * l + w1 * o.y;
+            m_ref = M;
+        }
+        const int slot = S == 0 ? w.slot0 : w.slot1;
+        if (slot < 0) {
+            const float inv = 1.f / l;
+            w0 *= inv;
+            w1 *= inv;
+            uint4 *orow = valid ? reinterpret_cast<uint4 *>(p.out + (((long long)w.b * p.q_len + qi) * p.n_q + h) * 128) : nullptr;
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t a[32];
+                tmem_ld32(o_addr + ch * 32, a);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * w0);
+                if (both) {
+                    uint32_t b2[32];
+                    tmem_ld32(o_addr + 128 + ch * 32, b2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(fmaf(__uint_as_float(b2[i]), w1, __uint_as_float(a[i])));
+                }
+                if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 u;
+                        u.x = pack_bf16(__uint_as_float(a[8 * i + 0]), __uint_as_float(a[8 * i + 1]));
+                        u.y = pack_bf16(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3]));
+                        u.z = pack_bf16(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5]));
+                        u.w = pack_bf16(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7]));
+                        orow[ch * 4 + i] = u;
+                    }
+                }
+            }
+            if (valid && p.lse != nullptr)
+                p.lse[((long long)w.b * p.n_q + h) * p.q_len + qi] = m_ref * p.scale + logf(l);
+        } else {
+            p.partial_ml[(long long)slot * KVP_TILE_ROWS + t] = make_float2(m_ref, l);
+            uint4 *orow = reinterpret_cast<uint4 *>(p.partial_o + ((long long)slot * KVP_TILE_ROWS + t) * 128);
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t a[32];
+                tmem_ld32(o_addr + ch * 32, a);
+                tc_wait_ld();
+                if (both) {
+                    uint32_t b2[32];
+                    tmem_ld32(o_addr + 128 + ch * 32, b2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        a[i] = __float_as_uint(fmaf(__uint_as_float(b2[i]), w1, __uint_as_float(a[i]) * w0));
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) orow[ch * 8 + i] = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+            }
+        }
+        tc_fence_before();
+        mbar_arrive(c.bar(kOFree + S));
+        if (both) mbar_arrive(c.bar(kOFree + 1));
+    }
+}
+
+// ---- Q producer -----------------------------------------------------------------------------------------
+__device__ __forceinline__ void producer_role(const Params &p, const Cta &c, const int t)
+{
+    uint32_t nEp0 = 0, nEp1 = 0;
+    bool ok = true;
+    for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
+        const Work w = load_work(p, wi);
+        const int n_rows = p.group * p.q_len;
+        const int max_steps = max(w.steps0, w.steps1);
+        int prev0 = 0, prev1 = 0;
+        auto produce = [&](int s, int rope, uint32_t &nEp) {
+            if (nEp > 0) {
+                ok = mbar_wait(c.bar(kQFree + s), (nEp - 1) & 1, c.abort_flag, p.status, 40 + s);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) return;
+            }
+            const int r = w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0) + t;
+            const __nv_bfloat16 *qrow = nullptr;
+            if (r < n_rows)
+                qrow = p.q + (((long long)w.b * p.q_len + r / p.group) * p.n_q + w.hk * p.group + r % p.group) * 128;
+            produce_q_row(p, c.smem + kOffQ + s * kTileBytes, t, qrow, rope);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(c.bar(kQFull + s));
+            ++nEp;
+        };
+        for (int k = 0; k < max_steps && ok; ++k) {
+            if (k < w.steps0) {
+                const int rope = get_tile(p, w, stream_tile(w, 0, k)).rope;
+                if (k == 0 || rope != prev0) produce(0, rope, nEp0);
+                prev0 = rope;
+            }
+            if (ok && k < w.steps1) {
+                const int rope = get_tile(p, w, stream_tile(w, 1, k)).rope;
+                if (k == 0 || rope != prev1) produce(1, rope, nEp1);
+                prev1 = rope;
+            }
+        }
+    }
+}
+
+// ---- TMA producer (whole warp; lane 0 issues) ----------------------------------------------------------
+__device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const int lane, const CUtensorMap *tm_pool_k,
+                                         const CUtensorMap *tm_pool_v, const CUtensorMap *tm_ws_k,
+                                         const CUtensorMap *tm_ws_v)
+{
+    uint32_t ring_n = 0;                                   // loads issued before this piece
+    bool ok = true;
+    for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
+        const Work w = load_work(p, wi);
+        const int n_loads = 2 * w.n;
+        for (int q0 = 0; q0 < n_loads && ok; q0 += 32) {
+            // lane i looks up the tile of load q0 + i
+            const int q = q0 + lane;
+            int r = 0, kv = 0;
+            if (w.mode == 0) { r = q >> 1; kv = q & 1; }
+            else if (q == 0) { r = 0; kv = 0; }
+            else if (q == n_loads - 1) { r = w.n - 1; kv = 1; }
+            else if (q & 1) { r = (q + 1) >> 1; kv = 0; }
+            else { r = (q - 2) >> 1; kv = 1; }
+            int row0 = 0, src = 0;
+            if (q < n_loads) {
+                const Tile tl = get_tile(p, w, w.lo + r);
+                row0 = tl.row0;
+                src = tl.src;
+            }
+            const int cnt = min(32, n_loads - q0);
+            for (int i = 0; i < cnt && ok; ++i) {
+                const int row0_i = __shfl_sync(0xffffffffu, row0, i);
+                const int src_i = __shfl_sync(0xffffffffu, src, i);
+                const int kv_i = __shfl_sync(0xffffffffu, kv, i);
+                if (lane == 0) {
+                    const uint32_t g = ring_n + (uint32_t)(q0 + i);
+                    const uint32_t stage = g % kStages, use = g / kStages;
+                    if (use > 0) ok = mbar_wait(c.bar(kKvEmpty + stage), (use - 1) & 1, c.abort_flag, p.status, 10 + stage);
+                    if (ok) {
+                        const CUtensorMap *tm = src_i == 0 ? (kv_i ? tm_pool_v : tm_pool_k) : (kv_i ? tm_ws_v : tm_ws_k);
+                        const uint32_t dst = c.smem_base + kOffRing + stage * kTileBytes;
+                        mbar_expect_tx(c.bar(kKvFull + stage), kTileBytes);
+                        tma_load_3d(dst, tm, 0, row0_i, w.plane, c.bar(kKvFull + stage));
+                        tma_load_3d(dst + kHalfBytes, tm, 64, row0_i, w.plane, c.bar(kKvFull + stage));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            }
+        }
+        ring_n += (uint32_t)n_loads;
+    }
+}
+
+// ---- MMA issuer (one thread) ----------------------------------------------------------------------------
+struct MmaStream {
+    uint32_t nP, nEpoch, nItems;
+    int prev_rope, prev_keys;
+    Tile cur, nxt;
+};
+
+__device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
+{
+    const uint32_t idesc_pv = instr_desc(128, 1);
+    MmaStream st[2];
+    st[0].nP = st[0].nEpoch = st[0].nItems = 0;
+    st[1].nP = st[1].nEpoch = st[1].nItems = 0;
+    uint32_t ring_n = 0;
+    bool ok = true;
+
+    for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
+        const Work w = load_work(p, wi);
+        const int steps[2] = {w.steps0, w.steps1};
+        const int max_steps = max(w.steps0, w.steps1);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            st[s].prev_rope = 0;
+            st[s].prev_keys = 0;
+            if (steps[s] > 0) st[s].cur = get_tile(p, w, stream_tile(w, s, 0));
+            if (steps[s] > 1) st[s].nxt = get_tile(p, w, stream_tile(w, s, 1));
+            else st[s].nxt = st[s].cur;
+        }
+        auto block = [&](auto s_c, int k) {
+            constexpr int s = decltype(s_c)::value;
+            MmaStream &ms = st[s];
+            const bool shared_stage = (w.mode == 0);              // mode 0: both streams read the same K/V stage
+            if (k >= 1 && k <= steps[s]) {
+                // ---- O_s += P_s V of step k-1 -------------------------------------------------------
+                const int r = w.mode ? 2 * (k - 1) + s : k - 1;
+                const uint32_t g = ring_n + (uint32_t)load_seq(w.mode, w.n, r, 1);
+                const uint32_t stage = g % kStages, par = (g / kStages) & 1;
+                if (!(shared_stage && s == 1)) ok = mbar_wait(c.bar(kKvFull + stage), par, c.abort_flag, p.status, 23);
+                if (ok) ok = mbar_wait(c.bar(kPFull + s), ms.nP & 1, c.abort_flag, p.status, 24 + s);
+                ++ms.nP;
+                if (ok && k == 1 && ms.nItems > 0)
+                    ok = mbar_wait(c.bar(kOFree + s), (ms.nItems - 1) & 1, c.abort_flag, p.status, 26 + s);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t va = c.smem_base + kOffRing + stage * kTileBytes;
+                const uint32_t pa = c.tmem + kColS + s * 128;
+                const uint32_t oa = c.tmem + kColO + s * 128;
+                const int ksteps = (ms.prev_keys + 15) >> 4;
+                for (int kk = 0; kk < ksteps; ++kk)
+                    mma_ts(oa, pa + kk * 8, smem_desc(va + kk * 2048, kHalfBytes), idesc_pv, (k > 1 || kk > 0));
+                if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
+                if (k == steps[s]) {
+                    tc_commit(c.bar(kOFull + s));
+                    ++ms.nItems;
+                }
+            }
+            if (k < steps[s]) {
+                // ---- S_s = Q_s K^T of step k -------------------------------------------------------------
+                const Tile tl = ms.cur;
+                if (k == 0 || tl.rope != ms.prev_rope) {
+                    ok = mbar_wait(c.bar(kQFull + s), ms.nEpoch & 1, c.abort_flag, p.status, 20 + s);
+                    ++ms.nEpoch;
+                }
+                const int r = w.mode ? 2 * k + s : k;
+                const uint32_t g = ring_n + (uint32_t)load_seq(w.mode, w.n, r, 0);
+                const uint32_t stage = g % kStages, par = (g / kStages) & 1;
+                if (ok && !(shared_stage && s == 1)) ok = mbar_wait(c.bar(kKvFull + stage), par, c.abort_flag, p.status, 22);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
+                const uint32_t idesc = instr_desc(n16, 0);
+                const uint32_t qa = c.smem_base + kOffQ + s * kTileBytes;
+                const uint32_t ka = c.smem_base + kOffRing + stage * kTileBytes;
+                const uint32_t d = c.tmem + kColS + s * 128;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    mma_ss(d, smem_desc(qa + off, 16), smem_desc(ka + off, 16), idesc, kk > 0);
+                }
+                tc_commit(c.bar(kSFull + s));
+                if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
+                const bool last = (k + 1 == steps[s]) || (ms.nxt.rope != tl.rope);
+                if (last) tc_commit(c.bar(kQFree + s));
+                ms.prev_rope = tl.rope;
+                ms.prev_keys = tl.n_keys;
+                ms.cur = ms.nxt;
+                if (k + 2 < steps[s]) ms.nxt = get_tile(p, w, stream_tile(w, s, k + 2));
+            }
+        };
+        for (int k = 0; k <= max_steps && ok; ++k) {
+            block(std::integral_constant<int, 0>{}, k);
+            if (ok) block(std::integral_constant<int, 1>{}, k);
+        }
+        ring_n += 2u * (uint32_t)w.n;
+    }
+    if (!ok) {                      // drain whatever was issued before giving TMEM back
+        tc_commit(c.bar(kDrain));
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(c.bar(kDrain), 0) && global_ns() - t0 < 100000000ull) {}
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_constant__ CUtensorMap tm_pool_v,
                   const __grid_constant__ CUtensorMap tm_ws_k, const __grid_constant__ CUtensorMap tm_ws_v,
                   const Params p)
 {
     extern __shared__ char smem_raw[];
-    char *smem = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t bar0 = smem_base + kOffBar;
-    auto bar = [&](int i) { return bar0 + 8u * i; };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffBar + 8 * kNumBars);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
+    Cta c;
+    c.smem = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    c.smem_base = smem_u32(c.smem);
+    c.bar0 = c.smem_base + kOffBar;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(c.smem + kOffBar + 8 * kNumBars);
+    c.abort_flag = tmem_slot + 1;
+    c.item_begin = __ldg(p.cta_begin + blockIdx.x);
+    c.item_end = __ldg(p.cta_begin + blockIdx.x + 1);
+    if (c.item_begin >= c.item_end) return;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- which unit of work --------------------------------------------------------------------
-    int x = blockIdx.x;
-    const int split = x % p.n_splits;  x /= p.n_splits;
-    const int mt = x % p.n_mtiles;     x /= p.n_mtiles;
-    const int hk = x % p.n_kv;
-    const int b = x / p.n_kv;
-    const kvp_item it = p.plan.items[b];
-    const int n_rows = p.group * p.q_len;
-    const int row_base = mt * KVP_TILE_ROWS;
-    const int i_max = min(n_rows - 1, row_base + KVP_TILE_ROWS - 1) / p.group;
-    const int n_tail = i_max / KVP_TILE_KEYS + 1;
-    const int n_all = n_tail + (it.tile_end - it.tile_begin);
-    const int lo = (int)((long long)n_all * split / p.n_splits);
-    const int n_my = (int)((long long)n_all * (split + 1) / p.n_splits) - lo;
-    const int plane = p.layer * p.n_kv + hk;
-    const long long unit = (long long)blockIdx.x;
-
-    if (n_my <= 0) {                       // nothing to do for this split: an empty partial
-        if (tid < KVP_TILE_ROWS && p.n_splits > 1) {
-            p.partial_ml[unit * KVP_TILE_ROWS + tid] = make_float2(-1e30f, 0.f);
-            float4 *o = reinterpret_cast<float4 *>(p.partial_o + (unit * KVP_TILE_ROWS + tid) * 128);
-            for (int c = 0; c < 32; ++c) o[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        return;
-    }
-
-    // ---- set-up --------------------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar(kKvFull + s), 1);
-            mbar_init(bar(kKvEmpty + s), 1);
+            mbar_init(c.bar(kKvFull + s), 1);
+            mbar_init(c.bar(kKvEmpty + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kQFull + s), 128);
-            mbar_init(bar(kSFull + s), 1);
-            mbar_init(bar(kPFull + s), 128);
-            mbar_init(bar(kPvDone + s), 1);
+            mbar_init(c.bar(kQFull + s), 128);
+            mbar_init(c.bar(kQFree + s), 1);
+            mbar_init(c.bar(kSFull + s), 1);
+            mbar_init(c.bar(kPFull + s), 128);
+            mbar_init(c.bar(kOFull + s), 1);
+            mbar_init(c.bar(kOFree + s), 128);
         }
-        mbar_init(bar(kDrain), 1);
-        *abort_flag = 0;
+        mbar_init(c.bar(kMlFull), 128);
+        mbar_init(c.bar(kDrain), 1);
+        *c.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == 12) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
                      "r"(kTmemCols)
                      : "memory");
@@ -351,246 +791,76 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
+    c.tmem = *tmem_slot;
 
-    if (warp == 4) {
-        // ================================ TMA producer ==========================================
-        if (lane == 0) {
-            for (int j = 0; j < n_my; ++j) {
-                const Tile tl = get_tile(p, it, n_tail, lo + j);
-                bool ok = true;
-                for (int kv = 0; kv < 2 && ok; ++kv) {
-                    const int n = 2 * j + kv, stage = n % kStages, use = n / kStages;
-                    if (use > 0) ok = mbar_wait(bar(kKvEmpty + stage), (use - 1) & 1, abort_flag, p.status, 10 + stage);
-                    if (!ok) break;
-                    const CUtensorMap *tm = tl.src == 0 ? (kv ? &tm_pool_v : &tm_pool_k) : (kv ? &tm_ws_v : &tm_ws_k);
-                    const uint32_t dst = smem_base + kOffRing + stage * kTileBytes;
-                    mbar_expect_tx(bar(kKvFull + stage), kTileBytes);
-                    tma_load_3d(dst, tm, 0, tl.row0, plane, bar(kKvFull + stage));
-                    tma_load_3d(dst + kHalfBytes, tm, 64, tl.row0, plane, bar(kKvFull + stage));
-                }
-                if (!ok) break;
-            }
-        }
-    } else if (warp == 5) {
-        // ================================ MMA issuer ============================================
-        if (lane == 0) {
-            const uint32_t idesc_pv = instr_desc(128, 1);
-            int ep = 0, prev_rope = 0;
-            bool ok = true;
-            auto issue_qk = [&](int j) {
-                const Tile tl = get_tile(p, it, n_tail, lo + j);
-                bool fresh = (j == 0);
-                if (j > 0 && tl.rope != prev_rope) { ++ep; fresh = true; }
-                prev_rope = tl.rope;
-                if (fresh) ok = mbar_wait(bar(kQFull + (ep & 1)), (ep >> 1) & 1, abort_flag, p.status, 20);
-                const int n = 2 * j, stage = n % kStages, sb = j & 1;
-                if (ok) ok = mbar_wait(bar(kKvFull + stage), (n / kStages) & 1, abort_flag, p.status, 21);
-                if (ok && j >= 2) ok = mbar_wait(bar(kPvDone + sb), ((j - 2) >> 1) & 1, abort_flag, p.status, 22);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
-                const uint32_t idesc = instr_desc(n16, 0);
-                const uint32_t qa = smem_base + kOffQ + (ep & 1) * kTileBytes;
-                const uint32_t ka = smem_base + kOffRing + stage * kTileBytes;
-                const uint32_t d = tmem + (sb ? kColS1 : kColS0);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                    mma_ss(d, smem_desc(qa + off, 16), smem_desc(ka + off, 16), idesc, k > 0);
-                }
-                tc_commit(bar(kKvEmpty + stage));
-                tc_commit(bar(kSFull + sb));
-            };
-            auto issue_pv = [&](int j) {
-                const Tile tl = get_tile(p, it, n_tail, lo + j);
-                const int n = 2 * j + 1, stage = n % kStages, sb = j & 1;
-                ok = mbar_wait(bar(kKvFull + stage), (n / kStages) & 1, abort_flag, p.status, 23);
-                if (ok) ok = mbar_wait(bar(kPFull + sb), (j >> 1) & 1, abort_flag, p.status, 24);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t va = smem_base + kOffRing + stage * kTileBytes;
-                const uint32_t pa = tmem + (sb ? kColS1 : kColS0);
-                const int ksteps = (tl.n_keys + 15) >> 4;
-                for (int k = 0; k < ksteps; ++k)
-                    mma_ts(tmem + kColO, pa + k * 8, smem_desc(va + k * 2048, kHalfBytes), idesc_pv, (j > 0 || k > 0));
-                tc_commit(bar(kKvEmpty + stage));
-                tc_commit(bar(kPvDone + sb));
-            };
-            issue_qk(0);
-            for (int j = 0; j < n_my && ok; ++j) {
-                if (j + 1 < n_my) issue_qk(j + 1);
-                if (ok) issue_pv(j);
-            }
-            if (!ok) {                      // drain whatever was issued before giving TMEM back
-                tc_commit(bar(kDrain));
-                const uint64_t t0 = global_ns();
-                while (!mbar_try_wait(bar(kDrain), 0) && global_ns() - t0 < 100000000ull) {}
-            }
-        }
+    if (warp < 4) {
+        reg_inc<kRegsSoftmax>();
+        softmax_role<0>(p, c, tid);
+    } else if (warp < 8) {
+        reg_inc<kRegsSoftmax>();
+        softmax_role<1>(p, c, tid - 128);
+    } else if (warp < 12) {
+        reg_dec<kRegsProducer>();
+        producer_role(p, c, tid - 256);
     } else {
-        // ================================ softmax / correction / epilogue ========================
-        const int r = row_base + tid;
-        const bool valid = r < n_rows;
-        const int qi = valid ? r / p.group : p.q_len - 1;
-        const int h = hk * p.group + (valid ? r % p.group : 0);
-        const __nv_bfloat16 *qrow = valid ? p.q + (((long long)b * p.q_len + qi) * p.n_q + h) * 128 : nullptr;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        const float c2 = p.scale_log2;
-
-        int ep = 0, prev_rope = 0;
-        {
-            const Tile t0 = get_tile(p, it, n_tail, lo);
-            prev_rope = t0.rope;
-            produce_q_row(p, smem + kOffQ, tid, qrow, t0.rope);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(bar(kQFull + 0));
-        }
-        float m_ref = -1e30f, l = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_my && ok; ++j) {
-            const Tile tl = get_tile(p, it, n_tail, lo + j);
-            const int sb = j & 1;
-            bool fresh = (j == 0);
-            if (j > 0 && tl.rope != prev_rope) { ++ep; fresh = true; }
-            prev_rope = tl.rope;
-            ok = mbar_wait(bar(kSFull + sb), (j >> 1) & 1, abort_flag, p.status, 30);
-            if (!ok) break;
-            tc_fence_after();
-            if (fresh) {
-                // first tile of a rotation epoch: prepare the next epoch's Q in the other buffer
-                // (its previous user's QK^T MMAs have all completed by now)
-                int nxt = -1;
-                for (int jj = j + 1; jj < n_my; ++jj) {
-                    const int rp = get_tile(p, it, n_tail, lo + jj).rope;
-                    if (rp != tl.rope) { nxt = rp; break; }
-                }
-                if (nxt >= 0) {
-                    produce_q_row(p, smem + kOffQ + ((ep + 1) & 1) * kTileBytes, tid, qrow, nxt);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    mbar_arrive(bar(kQFull + ((ep + 1) & 1)));
-                }
-            }
-            const uint32_t s_addr = tmem + lane_base + (sb ? kColS1 : kColS0);
-            const int n_chunks = (tl.n_keys + 31) >> 5;
-            const bool full = (tl.n_keys == KVP_TILE_KEYS) && (tl.qoff < 0);
-            const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);   // visible keys: [0, lim)
-
-            // pass 1: row max
-            float mx = -INFINITY;
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + ch * 32, v);
-                tc_wait_ld();
-                if (full) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (ch * 32 + c < lim) mx = fmaxf(mx, __uint_as_float(v[c]));
-                }
-            }
-            const float m_new = fmaxf(m_ref, mx);
-            if (j == 0) {
-                m_ref = m_new;
-            } else {
-                const bool need = (m_new - m_ref) * c2 > 8.0f;
-                if (__any_sync(0xffffffffu, need)) {
-                    // O is about to change scale: the previous P V product must have landed first
-                    ok = mbar_wait(bar(kPvDone + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, p.status, 31);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const float alpha = ex2((m_ref - m_new) * c2);
-                    m_ref = m_new;
-                    l *= alpha;
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t v[32];
-                        tmem_ld32(tmem + lane_base + kColO + ch * 32, v);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) v[c] = __float_as_uint(__uint_as_float(v[c]) * alpha);
-                        tmem_st32(tmem + lane_base + kColO + ch * 32, v);
-                    }
-                }
-            }
-            // pass 2: p = exp2((s - m) c), written over S as packed bf16 (chunk ch -> columns 16ch..16ch+15)
-            const float mc = m_ref * c2;
-            float lsum = 0.f;
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                uint32_t v[32], w[16];
-                tmem_ld32(s_addr + ch * 32, v);
-                tc_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(v[c]), c2, -mc));
-                    float p1 = ex2(fmaf(__uint_as_float(v[c + 1]), c2, -mc));
-                    if (!full) {
-                        if (ch * 32 + c >= lim) p0 = 0.f;
-                        if (ch * 32 + c + 1 >= lim) p1 = 0.f;
-                    }
-                    lsum += p0 + p1;
-                    w[c >> 1] = pack_bf16(p0, p1);
-                }
-                tmem_st16(s_addr + ch * 16, w);
-            }
-            l += lsum;
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(kPFull + sb));
-        }
-
-        if (ok) ok = mbar_wait(bar(kPvDone + ((n_my - 1) & 1)), ((n_my - 1) >> 1) & 1, abort_flag, p.status, 32);
-        ok = __all_sync(0xffffffffu, ok);
-        if (ok) {
-            tc_fence_after();
-            if (p.n_splits == 1) {
-                const float inv = 1.f / l;
-                uint4 *orow = valid ? reinterpret_cast<uint4 *>(p.out + (((long long)b * p.q_len + qi) * p.n_q + h) * 128) : nullptr;
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_base + kColO + ch * 32, v);
-                    tc_wait_ld();
-                    if (valid) {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint4 u;
-                            u.x = pack_bf16(__uint_as_float(v[8 * c + 0]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
-                            u.y = pack_bf16(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
-                            u.z = pack_bf16(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
-                            u.w = pack_bf16(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
-                            orow[ch * 4 + c] = u;
-                        }
-                    }
-                }
-                if (valid && p.lse != nullptr)
-                    p.lse[((long long)b * p.n_q + h) * p.q_len + qi] = m_ref * p.scale + logf(l);
-            } else {
-                p.partial_ml[unit * KVP_TILE_ROWS + tid] = make_float2(m_ref, l);
-                uint4 *orow = reinterpret_cast<uint4 *>(p.partial_o + (unit * KVP_TILE_ROWS + tid) * 128);
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_base + kColO + ch * 32, v);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) orow[ch * 8 + c] = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-                }
-            }
+        reg_dec<kRegsIssue>();
+        if (warp == 12) {
+            if (lane == 0) mma_role(p, c);
+        } else if (warp == 13) {
+            tma_role(p, c, lane, &tm_pool_k, &tm_pool_v, &tm_ws_k, &tm_ws_v);
         }
     }
 
     // ---- teardown ------------------------------------------------------------------------------
-    if (*abort_flag) {                      // let copies still in flight land before the CTA goes away
+    if (*c.abort_flag) {                    // let copies still in flight land before the CTA goes away
         const uint64_t t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 12) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+// ---- merge of the partial slots of split units ------------------------------------------------------------
+// Partials hold, per (slot, row): un-normalised O (fp32), the running max m of the raw scores and the
+// sum l of exp2((s - m) * c).  Block = 8 rows x 32 float4 columns; grid (merge item, 16).
+__global__ void __launch_bounds__(256)
+merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q, int group, float scale,
+                  const float *__restrict__ part_o, const float2 *__restrict__ part_ml,
+                  __nv_bfloat16 *__restrict__ out, float *__restrict__ lse)
+{
+    const kvp_merge_item mi = merges[blockIdx.x];
+    const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
+    const int c4 = threadIdx.x & 31;
+    const int r = mi.row_base + row;
+    if (r >= group * q_len) return;
+    const float c2 = scale * 1.4426950408889634f;
+    float M = -INFINITY;
+    for (int s = 0; s < mi.n_slots; ++s) {
+        const float2 ml = part_ml[(long long)(mi.slot0 + s) * KVP_TILE_ROWS + row];
+        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+    }
+    float L = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < mi.n_slots; ++s) {
+        const long long base = (long long)(mi.slot0 + s) * KVP_TILE_ROWS + row;
+        const float2 ml = part_ml[base];
+        if (!(ml.y > 0.f)) continue;                    // an empty partial: nothing was visible to this row
+        const float w = exp2f((ml.x - M) * c2);
+        L += w * ml.y;
+        const float4 a = reinterpret_cast<const float4 *>(part_o + base * 128)[c4];
+        o.x += w * a.x; o.y += w * a.y; o.z += w * a.z; o.w += w * a.w;
+    }
+    const float inv = 1.f / L;
+    const int i = r / group, h = mi.hk * group + r % group;
+    uint2 u;
+    u.x = pack_bf16(o.x * inv, o.y * inv);
+    u.y = pack_bf16(o.z * inv, o.w * inv);
+    reinterpret_cast<uint2 *>(out + (((long long)mi.b * q_len + i) * n_q + h) * 128)[c4] = u;
+    if (c4 == 0 && lse != nullptr) lse[((long long)mi.b * n_q + h) * q_len + i] = M * scale + logf(L);
 }
 
 }  // namespace
@@ -600,31 +870,38 @@ cudaError_t kvp_attn_sm100_prepare(void)
     return cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
-cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn_sm100_args &a, const CUtensorMap &tm_pool_k,
+cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, const CUtensorMap &tm_pool_k,
                                   const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
-                                  const CUtensorMap &tm_ws_v, int32_t *ctas, cudaStream_t st)
+                                  const CUtensorMap &tm_ws_v, cudaStream_t st)
 {
     Params p;
     p.plan = a.plan;
-    p.batch = a.batch;
     p.q_len = a.q_len;
     p.layer = a.layer;
-    p.n_splits = a.n_splits;
-    p.n_mtiles = a.n_mtiles;
     p.n_q = sh.n_q_heads;
     p.n_kv = sh.n_kv_heads;
     p.group = sh.group;
     p.pairing = sh.pairing;
     p.scale = sh.scale;
     p.scale_log2 = sh.scale * 1.4426950408889634f;
+    p.cta_begin = a.cta_begin;
+    p.works = a.works;
     p.q = (const __nv_bfloat16 *)a.q;
     p.out = (__nv_bfloat16 *)a.out;
     p.lse = a.lse;
     p.partial_o = a.partial_o;
     p.partial_ml = a.partial_ml;
     p.status = a.status;
-    const int grid = a.batch * sh.n_kv_heads * a.n_mtiles * a.n_splits;
-    if (ctas) *ctas = grid;
-    attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_pool_k, tm_pool_v, tm_ws_k, tm_ws_v, p);
+    attn_sm100_kernel<<<a.n_ctas, kThreads, kSmemBytes, st>>>(tm_pool_k, tm_pool_v, tm_ws_k, tm_ws_v, p);
+    return cudaGetLastError();
+}
+
+cudaError_t kvp_launch_merge_list(const kvp_shape &sh, int32_t q_len, int32_t n_merges, const kvp_merge_item *merges,
+                                  const float *partial_o, const float2 *partial_ml, void *out, float *lse,
+                                  cudaStream_t st)
+{
+    if (n_merges <= 0) return cudaSuccess;
+    merge_list_kernel<<<dim3(n_merges, KVP_TILE_ROWS / 8), 256, 0, st>>>(merges, q_len, sh.n_q_heads, sh.group, sh.scale,
+                                                                        partial_o, partial_ml, (__nv_bfloat16 *)out, lse);
     return cudaGetLastError();
 }

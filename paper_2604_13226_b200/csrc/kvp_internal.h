@@ -50,6 +50,29 @@ struct kvp_item {              // one request of the batch
     int32_t pad;
 };
 
+// One piece of work of the two-stream attention kernel: a contiguous range of one unit's key tiles.
+// A unit is up to 256 packed query rows of one (request, kv head).  Its key tiles are numbered: the
+// causal tiles of the query's own keys first, then the request's prefix tiles in plan order.
+//   mode 0: two 128-row query tiles ("streams"), each visiting every key tile of the range;
+//   mode 1: one 128-row query tile; the key tiles alternate between the two streams and the two
+//           partial results are combined inside the CTA.
+// slot >= 0: un-normalised fp32 partial written to that partial slot (the unit's key range is shared
+// by several pieces); slot < 0: this piece covers the whole range and writes the output rows.
+struct kvp_work {
+    int32_t b, hk;
+    int32_t row_base;          // first packed query row of the unit
+    int32_t mode;
+    int32_t tile_lo, n_tiles;  // range in the unit's tile numbering
+    int32_t slot0, slot1;      // stream 0 / stream 1 (mode 1 uses slot0 only)
+};
+
+struct kvp_merge_item {        // 128 packed rows whose result is spread over n_slots partial slots
+    int32_t b, hk;
+    int32_t row_base;
+    int32_t slot0, n_slots;
+    int32_t pad[3];
+};
+
 // Offsets (bytes) of the arrays inside one plan blob; identical on host and device.
 struct kvp_plan_layout {
     uint64_t items, tiles, chunks, segs, rope, total;
@@ -85,6 +108,8 @@ struct kvp_assembly_host {
     std::vector<kvp_tile> tiles;
     int32_t n_chunks = 0, n_rope = 0;
     int32_t last_q_len = 0;
+    // work list of the two-stream kernel, built for sched_q_len query tokens (0 = none yet)
+    int32_t sched_q_len = 0, sched_ctas = 0, sched_works = 0, sched_merges = 0, sched_slots = 0;
 };
 
 struct kvp_ctx {
@@ -102,6 +127,12 @@ struct kvp_ctx {
     kvp_plan_layout pl;
     std::vector<char *> slot_plan_dev;     // per assembly slot
     std::vector<char *> slot_k, slot_v;    // per assembly slot: workspace rows
+    std::vector<char *> slot_sched_dev;    // per assembly slot: cta ranges, work list, merge list
+    std::vector<char *> slot_sched_host;   // pinned staging of the same
+    std::vector<cudaEvent_t> sched_event;
+    uint64_t sched_off_works = 0, sched_off_merges = 0, sched_bytes = 0;
+    int32_t sched_max_works = 0, sched_max_merges = 0;
+    int32_t kernel_variant = 0;            // 0: two-stream kernel, 1: single-tile kernel
     float *partial_o = nullptr;            // [units][128][head_dim]
     float2 *partial_ml = nullptr;          // [units][128] (running max, running sum)
     char *q_scratch = nullptr;
@@ -157,10 +188,30 @@ struct kvp_attn_sm100_args {
     float2 *partial_ml;
     int32_t *status;
 };
-cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn_sm100_args &a, const CUtensorMap &tm_pool_k,
-                                  const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
-                                  const CUtensorMap &tm_ws_v, int32_t *ctas, cudaStream_t st);
 cudaError_t kvp_launch_merge(const kvp_shape &sh, int32_t batch, int32_t q_len, int32_t n_splits, int32_t n_mtiles,
                              const float *partial_o, const float2 *partial_ml, void *out, float *lse,
                              cudaStream_t st);
+cudaError_t kvp_attn_sm100_single_prepare(void);
+cudaError_t kvp_launch_attn_sm100_single(const kvp_shape &sh, const kvp_attn_sm100_args &a, const CUtensorMap &tm_pool_k,
+                                         const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
+                                         const CUtensorMap &tm_ws_v, int32_t *ctas, cudaStream_t st);
+
+struct kvp_attn2_args {
+    kvp_plan_dev plan;
+    int32_t q_len, layer, n_ctas;
+    const int32_t *cta_begin;      // [n_ctas + 1] ranges into works
+    const kvp_work *works;
+    const void *q;
+    void *out;
+    float *lse;
+    float *partial_o;
+    float2 *partial_ml;
+    int32_t *status;
+};
 cudaError_t kvp_attn_sm100_prepare(void);
+cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, const CUtensorMap &tm_pool_k,
+                                  const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
+                                  const CUtensorMap &tm_ws_v, cudaStream_t st);
+cudaError_t kvp_launch_merge_list(const kvp_shape &sh, int32_t q_len, int32_t n_merges, const kvp_merge_item *merges,
+                                  const float *partial_o, const float2 *partial_ml, void *out, float *lse,
+                                  cudaStream_t st);

@@ -162,14 +162,48 @@ def test_config2_bf16(materialize, simple):
     sess.close()
 
 
-@pytest.mark.parametrize("splits", [1, 2, 3, 7])
-def test_config2_forced_splits(splits):
+@pytest.mark.parametrize("ctas", [1, 2, 5, 22, 148])
+@pytest.mark.parametrize("no_split", [False, True])
+def test_config2_cta_counts(ctas, no_split):
+    # the persistent kernel's work list cut for 1..148 CTAs: one CTA walking every piece in turn,
+    # units split into partial slots and merged, and cuts only between units
     wl = gen.config2()
     sess = Session(wl)
     sess.assemble()
+    sess.ctx.tune(kvp.TUNE_SPLIT_TARGET_CTAS, ctas)
+    sess.ctx.tune(kvp.TUNE_FORCE_SPLITS, 1 if no_split else 0)
+    check_attention(wl, sess)
+    ll = sess.ctx.last_launch()
+    assert ll["kind"] == 1 and ll["ctas"] <= ctas
+    if no_split:
+        assert ll["splits"] == 1 and ll["launches"] == 2
+    sess.close()
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+def test_config2_single_tile_kernel_forced_splits(splits):
+    wl = gen.config2()
+    sess = Session(wl)
+    sess.assemble()
+    sess.ctx.tune(kvp.TUNE_KERNEL_VARIANT, 1)
     sess.ctx.tune(kvp.TUNE_FORCE_SPLITS, splits)
     check_attention(wl, sess)
     assert sess.ctx.last_launch()["splits"] == splits
+    sess.close()
+
+
+@pytest.mark.parametrize("q_len,n_docs,ctas", [(16, 1, 1), (16, 4, 3), (32, 3, 148), (1, 2, 2), (20, 2, 1), (33, 2, 5)])
+def test_one_query_tile_units(q_len, n_docs, ctas):
+    # g * q_len <= 128 rows per kv head (or a last unit of that size): the two streams of a CTA take
+    # alternate key tiles of the same query tile and are combined inside the CTA; odd and even tile
+    # counts, pieces of a single tile, several pieces per CTA
+    shape = gen.ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
+    lens = [300, 1024, 129, 640][:n_docs]
+    wl = gen.make_workload(shape, lens, [[(p, 0) for p in range(n_docs)]], q_len=q_len, seed=21 + q_len)
+    sess = Session(wl)
+    sess.assemble()
+    sess.ctx.tune(kvp.TUNE_SPLIT_TARGET_CTAS, ctas)
+    check_attention(wl, sess)
     sess.close()
 
 
@@ -193,8 +227,10 @@ def test_qwen_like_group7_long_query():
     sess = Session(wl)
     sess.assemble()
     check_attention(wl, sess)
-    sess.ctx.tune(kvp.TUNE_FORCE_SPLITS, 4)
-    check_attention(wl, sess)
+    for ctas in (7, 1):
+        sess.ctx.tune(kvp.TUNE_SPLIT_TARGET_CTAS, ctas)
+        sess.assemble()                      # a new assembly: the work list is rebuilt for the new CTA count
+        check_attention(wl, sess)
     sess.close()
 
 

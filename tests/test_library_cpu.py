@@ -128,3 +128,74 @@ def test_assembly_ring_drops_old_ids():
     with pytest.raises(kvp.KvpError):
         ctx.export_plan(a0, 0)
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# work list of the persistent attention kernel: every key tile of every unit exactly once
+# ------------------------------------------------------------------------------------------------
+
+def _schedule_case(n_q, n_kv, lens, items, q_len):
+    shape = gen.ModelShape(1, n_q, n_kv, 128, "bf16", 500000.0)
+    wl = gen.make_workload(shape, lens, items, q_len=q_len, n_header=16, n_trailer=16, seed=1)
+    ctx = host_ctx(shape, wl)
+    aid, plen = ctx.assemble(wl.items, kvp.REBASE)
+    return ctx, aid, plen, shape
+
+
+@pytest.mark.parametrize("case", [
+    (32, 8, [1024] * 10, [[(i, 0) for i in range(10)]] * 4, 128),        # config-3 shape: two-tile units, split
+    (32, 8, [2048] * 8, [[(i, 0) for i in range(8)]], 16),                # 64 rows per kv head: mode 1 units
+    (28, 4, [300, 1000, 257, 640], [[(0, 0), (1, 0)], [(2, 0), (3, 0), (0, -1)]], 50),   # g = 7, ragged
+    (8, 8, [100], [[(0, 0)]], 1),                                          # decode-like: one row per head
+    (32, 8, [512] * 5, [[(i, 0) for i in range(5)]], 64),                 # config-2 shape: little work
+    (4, 4, [200, 3000], [[(0, 0)], [(1, 0), (0, 0)]], 700),               # g = 1, many query tiles
+])
+def test_schedule_covers_every_tile_once(case):
+    n_q, n_kv, lens, items, q_len = case
+    ctx, aid, plen, shape = _schedule_case(n_q, n_kv, lens, items, q_len)
+    cb, works, merges, n_slots = ctx.export_schedule(aid, q_len)
+    g = n_q // n_kv
+    n_rows = g * q_len
+    assert cb[0] == 0 and cb[-1] == len(works) and np.all(np.diff(cb) > 0) and len(cb) - 1 <= 148
+    # expected units and their tile counts, from the assembly's own description
+    covered = {}
+    for w in works:
+        b, hk, row_base, mode, lo, n, s0, s1 = (int(x) for x in w)
+        assert 0 <= b < len(items) and 0 <= hk < n_kv and row_base % 256 == 0 and 0 <= row_base < n_rows
+        assert mode == (1 if n_rows - row_base <= 128 else 0) and n >= 1 and lo >= 0
+        covered.setdefault((b, hk, row_base), []).append((lo, n, s0, s1, mode))
+    slots_seen = []
+    for b in range(len(items)):
+        _, _, segs = ctx.export_plan(aid, b)
+        # prefix tiles: staged adapter rows form one run, each document its own run of <=128-key tiles
+        adapters = sum(int(s[1]) for s in segs if int(s[1]) in (16,) )
+        docs = [int(s[1]) for s in segs if int(s[1]) != 16]
+        n_prefix = -(-adapters // 128) + sum(-(-d // 128) for d in docs)
+        for hk in range(n_kv):
+            for row_base in range(0, n_rows, 256):
+                mode = 1 if n_rows - row_base <= 128 else 0
+                last = min(n_rows - 1, row_base + (128 if mode else 256) - 1)
+                n_all = (last // g) // 128 + 1 + n_prefix
+                pieces = sorted(covered.pop((b, hk, row_base)))
+                pos = 0
+                for lo, n, s0, s1, m in pieces:
+                    assert lo == pos
+                    pos += n
+                    if len(pieces) == 1:
+                        assert s0 == -1 and s1 == -1
+                    else:
+                        assert s0 >= 0 and (s1 >= 0) == (m == 0)
+                        slots_seen += [s0] + ([s1] if m == 0 else [])
+                assert pos == n_all
+    assert not covered
+    assert sorted(slots_seen) == list(range(n_slots))
+    # merge items name every slot exactly once, grouped per 128-row query tile
+    named = []
+    for m in merges:
+        b, hk, row_base, s0, n = (int(x) for x in m[:5])
+        assert n >= 2 and row_base % 128 == 0 and row_base < n_rows
+        named += list(range(s0, s0 + n))
+    assert sorted(named) == list(range(n_slots))
+    # balance: no CTA carries more than its share plus a few tiles
+    cost = [sum(int(works[i][5]) * (1 if works[i][3] else 2) for i in range(cb[c], cb[c + 1])) for c in range(len(cb) - 1)]
+    assert max(cost) <= sum(cost) / len(cost) + 8
