@@ -13,7 +13,8 @@
 //   warps 0-3 / 4-7   softmax of stream 0 / 1: one thread per query row.  S = Q K^T arrives in TMEM;
 //                     the thread takes the row max, forms p = exp2((s - m) * scale*log2e), sums it in
 //                     fp32, writes P as bf16 back into TMEM over S, and rescales O in TMEM when the
-//                     running max moved by more than 2^8.  At the end of a piece it normalises O and
+//                     running max moved by more than 2^8.  Both warpgroups run the same compact code
+//                     (rolled 32-column chunk loops) so that it stays in the instruction cache.  At the end of a piece it normalises O and
 //                     writes the output rows (or an fp32 partial when the unit's keys are split).
 //   warps 8-11        Q producer.  Documents keep the keys they were cached with: instead of rotating
 //                     every key by Delta (Eq. 1) the 128-row Q tile of a stream is counter-rotated by
@@ -46,8 +47,6 @@ constexpr int kOffBar = kOffRing + kStages * kTileBytes;
 constexpr int kOffMl = kOffBar + 256;                     // float2[128]: stream 1's (max, sum) in mode 1
 constexpr int kSmemBytes = kOffMl + 1024 + 1024;          // + alignment slack
 
-constexpr int kRegsSoftmax = 192, kRegsProducer = 72, kRegsIssue = 56;
-static_assert(2 * kRegsSoftmax + kRegsProducer + kRegsIssue <= 512, "register file");
 
 enum BarIdx { kKvFull = 0, kKvEmpty = kStages, kQFull = 2 * kStages, kQFree = kQFull + 2, kSFull = kQFree + 2,
               kPFull = kSFull + 2, kOFull = kPFull + 2, kOFree = kOFull + 2, kMlFull = kOFree + 2, kDrain = kMlFull + 1,
@@ -105,7 +104,7 @@ __device__ __forceinline__ uint64_t global_ns()
 
 // Bounded wait.  Returns false when another role has aborted or after ~2 s (then the status word and
 // the CTA's abort flag are set).  `code` identifies the wait.
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                             int32_t *status, int code)
 {
     const uint64_t t0 = global_ns();
@@ -215,8 +214,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
 //   K-major operand (Q, K): rows are 128-byte lines; the leading-dimension field is unused (1).
@@ -360,8 +357,45 @@ struct Cta {
 };
 
 // ---- softmax / correction / epilogue of stream S -------------------------------------------------------
-template <int S>
-__device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, const int t)
+// One thread per query row.  S is read from TMEM in 32-column chunks, twice (row max, then exponentials);
+// the chunk loops are rolled and shared by both streams so that the code stays resident in the
+// instruction cache; the next chunk is requested before the current one is processed.
+__device__ __forceinline__ float chunk_max(const uint32_t *v, float m)
+{
+    float m0 = m, m1 = m;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        m0 = fmax3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        m1 = fmax3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+    }
+    return fmaxf(m0, m1);
+}
+__device__ __forceinline__ void chunk_mask(uint32_t *v, int lim)
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (i >= lim) v[i] = 0xff800000u;                  // -inf
+}
+// p = exp2(s*c2 - mc) for 32 scores; packed bf16 to 16 TMEM columns; returns their fp32 sum
+__device__ __forceinline__ float chunk_exp_store(const uint32_t *v, float c2, float mc, uint32_t p_addr)
+{
+    uint32_t pk[16];
+    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float p0 = ex2(fmaf(__uint_as_float(v[i]), c2, -mc));
+        const float p1 = ex2(fmaf(__uint_as_float(v[i + 1]), c2, -mc));
+        const float p2 = ex2(fmaf(__uint_as_float(v[i + 2]), c2, -mc));
+        const float p3 = ex2(fmaf(__uint_as_float(v[i + 3]), c2, -mc));
+        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+        pk[i >> 1] = pack_bf16(p0, p1);
+        pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+    }
+    tmem_st16(p_addr, pk);
+    return (l0 + l1) + (l2 + l3);
+}
+
+__device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, const int S, const int t)
 {
     const uint32_t lane_base = (uint32_t)((t >> 5) * 32) << 16;
     const uint32_t s_addr = c.tmem + lane_base + kColS + S * 128;
@@ -383,6 +417,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
 
         float m_ref = -1e30f, l = 0.f;
         Tile nxt = get_tile(p, w, stream_tile(w, S, 0));
+#pragma unroll 1
         for (int k = 0; k < steps; ++k) {
             const Tile tl = nxt;
             if (k + 1 < steps) nxt = get_tile(p, w, stream_tile(w, S, k + 1));
@@ -392,32 +427,25 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
             if (!ok) break;
             tc_fence_after();
 
-            uint32_t v[128];
-            tmem_ld32(s_addr, v);
-            tmem_ld32(s_addr + 32, v + 32);
-            tmem_ld32(s_addr + 64, v + 64);
-            tmem_ld32(s_addr + 96, v + 96);
-            tc_wait_ld();
-
             const bool full = (tl.n_keys == KVP_TILE_KEYS) && (tl.qoff < 0);
-            if (!full) {
-                const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);   // visible keys: [0, lim)
-#pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i >= lim) v[i] = 0xff800000u;                                          // -inf
+            const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);       // visible keys: [0, lim)
+            uint32_t va[32], vb[32];
+
+            // pass 1: row max
+            float mx = -INFINITY;
+            tmem_ld32(s_addr, va);
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ch += 2) {
+                tc_wait_ld();
+                tmem_ld32(s_addr + (ch + 1) * 32, vb);
+                if (!full) chunk_mask(va, lim - ch * 32);
+                mx = chunk_max(va, mx);
+                tc_wait_ld();
+                tmem_ld32(s_addr + ((ch + 2) & 3) * 32, va);          // last round: chunk 0 again, for pass 2
+                if (!full) chunk_mask(vb, lim - (ch + 1) * 32);
+                mx = chunk_max(vb, mx);
             }
-            float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]), mx2 = __uint_as_float(v[2]),
-                  mx3 = __uint_as_float(v[3]);
-#pragma unroll
-            for (int i = 4; i < 124; i += 8) {
-                mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-                mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                mx2 = fmax3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-                mx3 = fmax3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-            }
-            mx0 = fmax3(mx0, __uint_as_float(v[124]), __uint_as_float(v[125]));
-            mx1 = fmax3(mx1, __uint_as_float(v[126]), __uint_as_float(v[127]));
-            const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
+            const float m_new = fmaxf(m_ref, mx);
             if (k == 0) {
                 m_ref = m_new;
             } else {
@@ -427,41 +455,30 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
                     const float alpha = need ? ex2((m_ref - m_new) * c2) : 1.f;
                     if (need) m_ref = m_new;
                     l *= alpha;
+                    tc_wait_ld();
 #pragma unroll 1
-                    for (int ch = 0; ch < 8; ++ch) {
-                        uint32_t o[16];
-                        asm volatile(
-                            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                            : KVP_R8(o, 0), KVP_R8(o, 8)
-                            : "r"(o_addr + ch * 16)
-                            : "memory");
+                    for (int ch = 0; ch < 4; ++ch) {
+                        tmem_ld32(o_addr + ch * 32, vb);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st16(o_addr + ch * 16, o);
+                        for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
+                        tmem_st32(o_addr + ch * 32, vb);
                     }
                 }
             }
-            // p = exp2((s - m) c), written over S as packed bf16 (columns 0..63 of the S block)
+            // pass 2: p = exp2((s - m) c), written over S as packed bf16 (columns 0..63 of the S block)
             const float mc = m_ref * c2;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    const float p0 = ex2(fmaf(__uint_as_float(v[ch * 32 + i]), c2, -mc));
-                    const float p1 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 1]), c2, -mc));
-                    const float p2 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 2]), c2, -mc));
-                    const float p3 = ex2(fmaf(__uint_as_float(v[ch * 32 + i + 3]), c2, -mc));
-                    l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                    pk[i >> 1] = pack_bf16(p0, p1);
-                    pk[(i >> 1) + 1] = pack_bf16(p2, p3);
-                }
-                tmem_st16(s_addr + ch * 16, pk);
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ch += 2) {
+                tc_wait_ld();
+                tmem_ld32(s_addr + (ch + 1) * 32, vb);
+                if (!full) chunk_mask(va, lim - ch * 32);
+                l += chunk_exp_store(va, c2, mc, s_addr + ch * 16);
+                tc_wait_ld();
+                if (ch == 0) tmem_ld32(s_addr + 64, va);
+                if (!full) chunk_mask(vb, lim - (ch + 1) * 32);
+                l += chunk_exp_store(vb, c2, mc, s_addr + (ch + 1) * 16);
             }
-            l += (l0 + l1) + (l2 + l3);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(c.bar(kPFull + S));
@@ -496,58 +513,49 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
             m_ref = M;
         }
         const int slot = S == 0 ? w.slot0 : w.slot1;
-        if (slot < 0) {
+        const bool direct = slot < 0;
+        if (direct) {
             const float inv = 1.f / l;
             w0 *= inv;
             w1 *= inv;
-            uint4 *orow = valid ? reinterpret_cast<uint4 *>(p.out + (((long long)w.b * p.q_len + qi) * p.n_q + h) * 128) : nullptr;
+        }
+        // un-normalised (partial slot) or normalised (output rows) O = w0 O_s (+ w1 O_1)
+        uint4 *orow_bf = (direct && valid) ? reinterpret_cast<uint4 *>(p.out + (((long long)w.b * p.q_len + qi) * p.n_q + h) * 128) : nullptr;
+        uint4 *orow_f = direct ? nullptr : reinterpret_cast<uint4 *>(p.partial_o + ((long long)slot * KVP_TILE_ROWS + t) * 128);
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t a[32];
-                tmem_ld32(o_addr + ch * 32, a);
+        for (int ch = 0; ch < 4; ++ch) {
+            uint32_t a[32];
+            tmem_ld32(o_addr + ch * 32, a);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * w0);
+            if (both) {
+                uint32_t b2[32];
+                tmem_ld32(o_addr + 128 + ch * 32, b2);
                 tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * w0);
-                if (both) {
-                    uint32_t b2[32];
-                    tmem_ld32(o_addr + 128 + ch * 32, b2);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(fmaf(__uint_as_float(b2[i]), w1, __uint_as_float(a[i])));
-                }
-                if (valid) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 u;
-                        u.x = pack_bf16(__uint_as_float(a[8 * i + 0]), __uint_as_float(a[8 * i + 1]));
-                        u.y = pack_bf16(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3]));
-                        u.z = pack_bf16(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5]));
-                        u.w = pack_bf16(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7]));
-                        orow[ch * 4 + i] = u;
-                    }
-                }
+                for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(fmaf(__uint_as_float(b2[i]), w1, __uint_as_float(a[i])));
             }
+            if (orow_bf != nullptr) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 u;
+                    u.x = pack_bf16(__uint_as_float(a[8 * i + 0]), __uint_as_float(a[8 * i + 1]));
+                    u.y = pack_bf16(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3]));
+                    u.z = pack_bf16(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5]));
+                    u.w = pack_bf16(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7]));
+                    orow_bf[ch * 4 + i] = u;
+                }
+            } else if (orow_f != nullptr) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) orow_f[ch * 8 + i] = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+            }
+        }
+        if (direct) {
             if (valid && p.lse != nullptr)
                 p.lse[((long long)w.b * p.n_q + h) * p.q_len + qi] = m_ref * p.scale + logf(l);
         } else {
             p.partial_ml[(long long)slot * KVP_TILE_ROWS + t] = make_float2(m_ref, l);
-            uint4 *orow = reinterpret_cast<uint4 *>(p.partial_o + ((long long)slot * KVP_TILE_ROWS + t) * 128);
-#pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t a[32];
-                tmem_ld32(o_addr + ch * 32, a);
-                tc_wait_ld();
-                if (both) {
-                    uint32_t b2[32];
-                    tmem_ld32(o_addr + 128 + ch * 32, b2);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        a[i] = __float_as_uint(fmaf(__uint_as_float(b2[i]), w1, __uint_as_float(a[i]) * w0));
-                }
-#pragma unroll
-                for (int i = 0; i < 8; ++i) orow[ch * 8 + i] = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-            }
         }
         tc_fence_before();
         mbar_arrive(c.bar(kOFree + S));
@@ -793,17 +801,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
     tc_fence_after();
     c.tmem = *tmem_slot;
 
-    if (warp < 4) {
-        reg_inc<kRegsSoftmax>();
-        softmax_role<0>(p, c, tid);
-    } else if (warp < 8) {
-        reg_inc<kRegsSoftmax>();
-        softmax_role<1>(p, c, tid - 128);
+    if (warp < 8) {
+        softmax_role(p, c, warp >> 2, tid & 127);
     } else if (warp < 12) {
-        reg_dec<kRegsProducer>();
         producer_role(p, c, tid - 256);
     } else {
-        reg_dec<kRegsIssue>();
         if (warp == 12) {
             if (lane == 0) mma_role(p, c);
         } else if (warp == 13) {
