@@ -145,13 +145,22 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// 64-bit shared-memory matrix descriptors are kept as a constant high word and a low word (start
+// address and leading-dimension offset, in 16-byte units) that advances by an immediate per K-step.
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc)
+template <int ACC>
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc)
+        ::"r"(d), "l"(a), "l"(b), "r"(idesc), "n"(ACC)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
@@ -161,6 +170,15 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint3
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc)
+        : "memory");
+}
+template <int ACC>
+__device__ __forceinline__ void mma_ts_c(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(b), "r"(idesc), "n"(ACC)
         : "memory");
 }
 
@@ -218,14 +236,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
 //   K-major operand (Q, K): rows are 128-byte lines; the leading-dimension field is unused (1).
 //   MN-major operand (V):   the second 64-column block lies `lbo_bytes` further on.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, sm_100 version, SWIZZLE_128B
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes)
 {
-    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;
-    d |= (uint64_t)(1024u >> 4) << 32;
-    d |= 1ull << 46;                    // descriptor version for sm_100
-    d |= 2ull << 61;                    // SWIZZLE_128B
-    return d;
+    return ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
 __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major)
@@ -297,54 +311,62 @@ __device__ __forceinline__ int load_seq(int mode, int n, int r, int kv)
     return r <= n - 2 ? 2 * r + 2 : 2 * n - 1;
 }
 
-// Write this thread's query row, counter-rotated by the offset of rope-table row `rope`, into a
-// rotated-Q buffer in the K-major 128-byte-swizzled layout (two 64-column halves of 128 x 128 bytes).
-__device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t, const __nv_bfloat16 *qrow, int rope)
+// This thread's query row (128 bf16 = 16 x 16 bytes), counter-rotated in registers by the offset of
+// rope-table row `rope`: q' = R(-Delta) q, which leaves q'.k = q.(R(Delta) k) (Eq. 1 moved onto Q).
+__device__ __forceinline__ void load_rotate_q_row(const Params &p, uint4 (&qv)[16], const __nv_bfloat16 *qrow, int rope)
+{
+    if (qrow == nullptr) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) qv[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) qv[c] = __ldg(src + c);
+    if (rope == 0) return;
+    const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
+    auto lo_f = [](uint32_t u) { return __uint_as_float(u << 16); };
+    auto hi_f = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
+    if (p.pairing == 0) {
+        // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint32_t *a = reinterpret_cast<uint32_t *>(&qv[c]);
+            uint32_t *b = reinterpret_cast<uint32_t *>(&qv[c + 8]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 w = __ldg(cs + c * 4 + j);                  // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
+                const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
+                a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
+                b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
+            }
+        }
+    } else {
+        // pairs (2i, 2i+1): one word each
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            uint32_t *a = reinterpret_cast<uint32_t *>(&qv[c]);
+#pragma unroll
+            for (int j = 0; j < 4; j += 2) {
+                const float4 w = __ldg(cs + c * 2 + (j >> 1));           // pairs 4c+j, 4c+j+1
+                const float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
+                a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+            }
+        }
+    }
+}
+// Store the row into a rotated-Q buffer in the K-major 128-byte-swizzled layout (two 64-column halves
+// of 128 rows x 128 bytes).
+__device__ __forceinline__ void store_q_row(char *qbuf, int t, const uint4 (&qv)[16])
 {
     const int sw = t & 7;
     char *row_lo = qbuf + t * 128;
     char *row_hi = row_lo + kHalfBytes;
-    if (qrow == nullptr) {
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
-        }
-        return;
-    }
-    const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
-    const float2 *cs = p.plan.rope + (size_t)rope * 64;
-#pragma unroll 2
     for (int c = 0; c < 8; ++c) {
-        union { uint4 u; __nv_bfloat16 e[8]; } lo, hi;
-        lo.u = __ldg(src + c);
-        hi.u = __ldg(src + c + 8);
-        if (rope != 0) {
-            if (p.pairing == 0) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float2 w = __ldg(cs + c * 8 + k);
-                    const float a = __bfloat162float(lo.e[k]), b = __bfloat162float(hi.e[k]);
-                    lo.e[k] = __float2bfloat16_rn(a * w.x + b * w.y);        // R(-Delta): cos same, sin negated
-                    hi.e[k] = __float2bfloat16_rn(b * w.x - a * w.y);
-                }
-            } else {
-#pragma unroll
-                for (int k = 0; k < 8; k += 2) {
-                    float2 w = __ldg(cs + (c * 8 + k) / 2);
-                    float a = __bfloat162float(lo.e[k]), b = __bfloat162float(lo.e[k + 1]);
-                    lo.e[k] = __float2bfloat16_rn(a * w.x + b * w.y);
-                    lo.e[k + 1] = __float2bfloat16_rn(b * w.x - a * w.y);
-                    w = __ldg(cs + ((c + 8) * 8 + k) / 2);
-                    a = __bfloat162float(hi.e[k]);
-                    b = __bfloat162float(hi.e[k + 1]);
-                    hi.e[k] = __float2bfloat16_rn(a * w.x + b * w.y);
-                    hi.e[k + 1] = __float2bfloat16_rn(b * w.x - a * w.y);
-                }
-            }
-        }
-        *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = lo.u;
-        *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = hi.u;
+        *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = qv[c];
+        *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = qv[c + 8];
     }
 }
 
@@ -574,16 +596,19 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
         auto produce = [&](int s, int rope, uint32_t &nEp) {
+            // the row is fetched and rotated while the previous document still uses the buffer
+            const int r = w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0) + t;
+            const __nv_bfloat16 *qrow = nullptr;
+            if (r < n_rows)
+                qrow = p.q + (((long long)w.b * p.q_len + r / p.group) * p.n_q + w.hk * p.group + r % p.group) * 128;
+            uint4 qv[16];
+            load_rotate_q_row(p, qv, qrow, rope);
             if (nEp > 0) {
                 ok = mbar_wait(c.bar(kQFree + s), (nEp - 1) & 1, c.abort_flag, p.status, 40 + s);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
             }
-            const int r = w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0) + t;
-            const __nv_bfloat16 *qrow = nullptr;
-            if (r < n_rows)
-                qrow = p.q + (((long long)w.b * p.q_len + r / p.group) * p.n_q + w.hk * p.group + r % p.group) * 128;
-            produce_q_row(p, c.smem + kOffQ + s * kTileBytes, t, qrow, rope);
+            store_q_row(c.smem + kOffQ + s * kTileBytes, t, qv);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(c.bar(kQFull + s));
             ++nEp;
@@ -696,12 +721,18 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                     ok = mbar_wait(c.bar(kOFree + s), (ms.nItems - 1) & 1, c.abort_flag, p.status, 26 + s);
                 if (!ok) return;
                 tc_fence_after();
-                const uint32_t va = c.smem_base + kOffRing + stage * kTileBytes;
+                const uint32_t v_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, kHalfBytes);
                 const uint32_t pa = c.tmem + kColS + s * 128;
                 const uint32_t oa = c.tmem + kColO + s * 128;
-                const int ksteps = (ms.prev_keys + 15) >> 4;
-                for (int kk = 0; kk < ksteps; ++kk)
-                    mma_ts(oa, pa + kk * 8, smem_desc(va + kk * 2048, kHalfBytes), idesc_pv, (k > 1 || kk > 0));
+                if (ms.prev_keys == KVP_TILE_KEYS && k > 1) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)               // 16 keys per step: P advances 8 columns, V 2048 bytes
+                        mma_ts_c<1>(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv);
+                } else {
+                    const int ksteps = (ms.prev_keys + 15) >> 4;
+                    for (int kk = 0; kk < ksteps; ++kk)
+                        mma_ts(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv, (k > 1 || kk > 0));
+                }
                 if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
                 if (k == steps[s]) {
                     tc_commit(c.bar(kOFull + s));
@@ -723,13 +754,15 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 tc_fence_after();
                 const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
                 const uint32_t idesc = instr_desc(n16, 0);
-                const uint32_t qa = c.smem_base + kOffQ + s * kTileBytes;
-                const uint32_t ka = c.smem_base + kOffRing + stage * kTileBytes;
+                const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + s * kTileBytes, 16);
+                const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
                 const uint32_t d = c.tmem + kColS + s * 128;
+                mma_ss<0>(d, desc64(q_lo, kDescHi), desc64(k_lo, kDescHi), idesc);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                    mma_ss(d, smem_desc(qa + off, 16), smem_desc(ka + off, 16), idesc, kk > 0);
+                for (int kk = 1; kk < 8; ++kk) {                 // 16 columns per step: 32 bytes, second half 16 KB on
+                    constexpr uint32_t kHalf16 = kHalfBytes >> 4;
+                    const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
+                    mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
                 }
                 tc_commit(c.bar(kSFull + s));
                 if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
