@@ -138,9 +138,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// The MMA warp runs convergently; one elected lane issues each tcgen05.mma / tcgen05.commit.
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -158,8 +161,8 @@ template <int ACC>
 __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d), "l"(a), "l"(b), "r"(idesc), "n"(ACC)
         : "memory");
 }
@@ -167,8 +170,8 @@ __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint3
 __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc)
         : "memory");
 }
@@ -176,8 +179,8 @@ template <int ACC>
 __device__ __forceinline__ void mma_ts_c(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d), "r"(a), "l"(b), "r"(idesc), "n"(ACC)
         : "memory");
 }
@@ -677,7 +680,7 @@ __device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const in
     }
 }
 
-// ---- MMA issuer (one thread) ----------------------------------------------------------------------------
+// ---- MMA issuer (whole warp, convergent; one elected lane issues) ----------------------------------------------------------------------------
 struct MmaStream {
     uint32_t nP, nEpoch, nItems;
     int prev_rope, prev_keys;
@@ -719,6 +722,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 ++ms.nP;
                 if (ok && k == 1 && ms.nItems > 0)
                     ok = mbar_wait(c.bar(kOFree + s), (ms.nItems - 1) & 1, c.abort_flag, p.status, 26 + s);
+                ok = __all_sync(0xffffffffu, ok);                 // the lanes stay together
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t v_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, kHalfBytes);
@@ -750,6 +754,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 const uint32_t g = ring_n + (uint32_t)load_seq(w.mode, w.n, r, 0);
                 const uint32_t stage = g % kStages, par = (g / kStages) & 1;
                 if (ok && !(shared_stage && s == 1)) ok = mbar_wait(c.bar(kKvFull + stage), par, c.abort_flag, p.status, 22);
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
@@ -780,6 +785,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
         }
         ring_n += 2u * (uint32_t)w.n;
     }
+    __syncwarp();
     if (!ok) {                      // drain whatever was issued before giving TMEM back
         tc_commit(c.bar(kDrain));
         const uint64_t t0 = global_ns();
@@ -840,7 +846,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
         producer_role(p, c, tid - 256);
     } else {
         if (warp == 12) {
-            if (lane == 0) mma_role(p, c);
+            mma_role(p, c);
         } else if (warp == 13) {
             tma_role(p, c, lane, &tm_pool_k, &tm_pool_v, &tm_ws_k, &tm_ws_v);
         }
