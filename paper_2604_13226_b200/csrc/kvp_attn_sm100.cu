@@ -18,10 +18,11 @@
 //                     writes the output rows (or an fp32 partial when the unit's keys are split).
 //   warps 8-11        Q producer.  Documents keep the keys they were cached with: instead of rotating
 //                     every key by Delta (Eq. 1) the 128-row Q tile of a stream is counter-rotated by
-//                     -Delta once per document, which leaves every score q.k unchanged.
+//                     -Delta once per document, which leaves every score q.k unchanged.  Each stream has
+//                     two Q buffers, so the next document's Q is written while the current one is in use.
 //   warp 12           MMA issuer and TMEM owner.  Per stream and step: O += P V of the previous tile,
 //                     then S = Q K^T of the next one; the two streams alternate.
-//   warp 13           TMA producer: K and V tiles into a 5-stage ring (two 64-column boxes each,
+//   warp 13           TMA producer: K and V tiles into a 3-stage ring (two 64-column boxes each,
 //                     128-byte swizzle), in the order the MMA warp consumes them.
 //
 // Every mbarrier wait is bounded: when it runs out the CTA records a code in the status word, drains
@@ -34,21 +35,21 @@
 
 namespace {
 
-constexpr int kStages = 5;
+constexpr int kStages = 3;
 constexpr int kTileBytes = KVP_TILE_KEYS * 128 * 2;      // 32 KB: 128 rows x 128 bf16
 constexpr int kHalfBytes = kTileBytes / 2;               // one 64-column box
 constexpr int kThreads = 512;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;               // + 128 * stream
 
-constexpr int kOffQ = 0;                                  // one 32 KB rotated-Q buffer per stream
-constexpr int kOffRing = 2 * kTileBytes;                  // kStages x 32 KB
+constexpr int kOffQ = 0;                                  // two 32 KB rotated-Q buffers per stream: [stream][epoch & 1]
+constexpr int kOffRing = 4 * kTileBytes;                  // kStages x 32 KB
 constexpr int kOffBar = kOffRing + kStages * kTileBytes;
 constexpr int kOffMl = kOffBar + 256;                     // float2[128]: stream 1's (max, sum) in mode 1
 constexpr int kSmemBytes = kOffMl + 1024 + 1024;          // + alignment slack
 
 
-enum BarIdx { kKvFull = 0, kKvEmpty = kStages, kQFull = 2 * kStages, kQFree = kQFull + 2, kSFull = kQFree + 2,
+enum BarIdx { kKvFull = 0, kKvEmpty = kStages, kQFull = 2 * kStages, kQFree = kQFull + 4, kSFull = kQFree + 4,   // Q: [2 * stream + buffer]
               kPFull = kSFull + 2, kOFull = kPFull + 2, kOFree = kOFull + 2, kMlFull = kOFree + 2, kDrain = kMlFull + 1,
               kNumBars = kDrain + 1 };
 static_assert(8 * kNumBars + 8 <= 256, "barrier block");
@@ -314,62 +315,58 @@ __device__ __forceinline__ int load_seq(int mode, int n, int r, int kv)
     return r <= n - 2 ? 2 * r + 2 : 2 * n - 1;
 }
 
-// This thread's query row (128 bf16 = 16 x 16 bytes), counter-rotated in registers by the offset of
-// rope-table row `rope`: q' = R(-Delta) q, which leaves q'.k = q.(R(Delta) k) (Eq. 1 moved onto Q).
-__device__ __forceinline__ void load_rotate_q_row(const Params &p, uint4 (&qv)[16], const __nv_bfloat16 *qrow, int rope)
-{
-    if (qrow == nullptr) {
-#pragma unroll
-        for (int c = 0; c < 16; ++c) qv[c] = make_uint4(0, 0, 0, 0);
-        return;
-    }
-    const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
-#pragma unroll
-    for (int c = 0; c < 16; ++c) qv[c] = __ldg(src + c);
-    if (rope == 0) return;
-    const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
-    auto lo_f = [](uint32_t u) { return __uint_as_float(u << 16); };
-    auto hi_f = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
-    if (p.pairing == 0) {
-        // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            uint32_t *a = reinterpret_cast<uint32_t *>(&qv[c]);
-            uint32_t *b = reinterpret_cast<uint32_t *>(&qv[c + 8]);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float4 w = __ldg(cs + c * 4 + j);                  // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
-                const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
-                a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
-                b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
-            }
-        }
-    } else {
-        // pairs (2i, 2i+1): one word each
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            uint32_t *a = reinterpret_cast<uint32_t *>(&qv[c]);
-#pragma unroll
-            for (int j = 0; j < 4; j += 2) {
-                const float4 w = __ldg(cs + c * 2 + (j >> 1));           // pairs 4c+j, 4c+j+1
-                const float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
-                a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
-                a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
-            }
-        }
-    }
-}
-// Store the row into a rotated-Q buffer in the K-major 128-byte-swizzled layout (two 64-column halves
-// of 128 rows x 128 bytes).
-__device__ __forceinline__ void store_q_row(char *qbuf, int t, const uint4 (&qv)[16])
+// Write this thread's query row (128 bf16 = 16 x 16 bytes), counter-rotated by the offset of rope-table
+// row `rope` - q' = R(-Delta) q, which leaves q'.k = q.(R(Delta) k), Eq. 1 moved onto Q - into a rotated-Q
+// buffer in the K-major 128-byte-swizzled layout (two 64-column halves of 128 rows x 128 bytes).
+__device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t, const __nv_bfloat16 *qrow, int rope)
 {
     const int sw = t & 7;
     char *row_lo = qbuf + t * 128;
     char *row_hi = row_lo + kHalfBytes;
+    if (qrow == nullptr) {
 #pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
+    const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
+    auto lo_f = [](uint32_t u) { return __uint_as_float(u << 16); };
+    auto hi_f = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
+#pragma unroll 2
     for (int c = 0; c < 8; ++c) {
-        *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = qv[c];
-        *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = qv[c + 8];
+        uint4 qa = __ldg(src + c), qb = __ldg(src + c + 8);
+        uint32_t *a = reinterpret_cast<uint32_t *>(&qa);
+        uint32_t *b = reinterpret_cast<uint32_t *>(&qb);
+        if (rope != 0) {
+            if (p.pairing == 0) {
+                // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 w = __ldg(cs + c * 4 + j);              // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
+                    const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
+                    a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
+                    b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
+                }
+            } else {
+                // pairs (2i, 2i+1): one word each; chunk c holds pairs 4c..4c+3
+#pragma unroll
+                for (int j = 0; j < 4; j += 2) {
+                    float4 w = __ldg(cs + c * 2 + (j >> 1));
+                    float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
+                    a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                    a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+                    w = __ldg(cs + (c + 8) * 2 + (j >> 1));
+                    x0 = lo_f(b[j]); y0 = hi_f(b[j]); x1 = lo_f(b[j + 1]); y1 = hi_f(b[j + 1]);
+                    b[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                    b[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+                }
+            }
+        }
+        *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = qa;
+        *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = qb;
     }
 }
 
@@ -599,21 +596,19 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
         auto produce = [&](int s, int rope, uint32_t &nEp) {
-            // the row is fetched and rotated while the previous document still uses the buffer
+            const int buf = nEp & 1;
+            if (nEp >= 2) {                                 // the epoch before last used this buffer
+                ok = mbar_wait(c.bar(kQFree + 2 * s + buf), ((nEp >> 1) - 1) & 1, c.abort_flag, p.status, 40 + s);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) return;
+            }
             const int r = w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0) + t;
             const __nv_bfloat16 *qrow = nullptr;
             if (r < n_rows)
                 qrow = p.q + (((long long)w.b * p.q_len + r / p.group) * p.n_q + w.hk * p.group + r % p.group) * 128;
-            uint4 qv[16];
-            load_rotate_q_row(p, qv, qrow, rope);
-            if (nEp > 0) {
-                ok = mbar_wait(c.bar(kQFree + s), (nEp - 1) & 1, c.abort_flag, p.status, 40 + s);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return;
-            }
-            store_q_row(c.smem + kOffQ + s * kTileBytes, t, qv);
+            produce_q_row(p, c.smem + kOffQ + (2 * s + buf) * kTileBytes, t, qrow, rope);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(c.bar(kQFull + s));
+            mbar_arrive(c.bar(kQFull + 2 * s + buf));
             ++nEp;
         };
         for (int k = 0; k < max_steps && ok; ++k) {
@@ -682,7 +677,7 @@ __device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const in
 
 // ---- MMA issuer (whole warp, convergent; one elected lane issues) ----------------------------------------------------------------------------
 struct MmaStream {
-    uint32_t nP, nEpoch, nItems;
+    uint32_t nP, nEpoch, nItems, qbuf;
     int prev_rope, prev_keys;
     Tile cur, nxt;
 };
@@ -691,8 +686,8 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
 {
     const uint32_t idesc_pv = instr_desc(128, 1);
     MmaStream st[2];
-    st[0].nP = st[0].nEpoch = st[0].nItems = 0;
-    st[1].nP = st[1].nEpoch = st[1].nItems = 0;
+    st[0].nP = st[0].nEpoch = st[0].nItems = st[0].qbuf = 0;
+    st[1].nP = st[1].nEpoch = st[1].nItems = st[1].qbuf = 0;
     uint32_t ring_n = 0;
     bool ok = true;
 
@@ -746,8 +741,9 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
             if (k < steps[s]) {
                 // ---- S_s = Q_s K^T of step k -------------------------------------------------------------
                 const Tile tl = ms.cur;
-                if (k == 0 || tl.rope != ms.prev_rope) {
-                    ok = mbar_wait(c.bar(kQFull + s), ms.nEpoch & 1, c.abort_flag, p.status, 20 + s);
+                if (k == 0 || tl.rope != ms.prev_rope) {            // first tile of a document: its own Q buffer
+                    ms.qbuf = ms.nEpoch & 1;
+                    ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
                     ++ms.nEpoch;
                 }
                 const int r = w.mode ? 2 * k + s : k;
@@ -759,7 +755,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 tc_fence_after();
                 const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
                 const uint32_t idesc = instr_desc(n16, 0);
-                const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + s * kTileBytes, 16);
+                const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
                 const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
                 const uint32_t d = c.tmem + kColS + s * 128;
                 mma_ss<0>(d, desc64(q_lo, kDescHi), desc64(k_lo, kDescHi), idesc);
@@ -772,7 +768,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 tc_commit(c.bar(kSFull + s));
                 if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
                 const bool last = (k + 1 == steps[s]) || (ms.nxt.rope != tl.rope);
-                if (last) tc_commit(c.bar(kQFree + s));
+                if (last) tc_commit(c.bar(kQFree + 2 * s + ms.qbuf));
                 ms.prev_rope = tl.rope;
                 ms.prev_keys = tl.n_keys;
                 ms.cur = ms.nxt;
@@ -816,9 +812,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
             mbar_init(c.bar(kKvFull + s), 1);
             mbar_init(c.bar(kKvEmpty + s), 1);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 4; ++s) {
             mbar_init(c.bar(kQFull + s), 128);
             mbar_init(c.bar(kQFree + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(c.bar(kSFull + s), 1);
             mbar_init(c.bar(kPFull + s), 128);
             mbar_init(c.bar(kOFull + s), 1);
