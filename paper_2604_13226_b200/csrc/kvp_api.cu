@@ -178,6 +178,10 @@ int find_slot(kvp_ctx *ctx, int32_t assembly_id)
 // rows of one request and kv head) are laid end to end, each weighted by the tensor-core work of its
 // key tiles, and the line is cut into equal shares, one per CTA; a cut closer than two tiles to a unit
 // boundary moves onto it.  A unit that ends up in several pieces gets partial slots and merge items.
+// Start-up and write-out of a piece (first Q tile, pipeline fill, epilogue) cost about as much as four
+// two-stream key tiles; the unit weights carry it so that CTAs with more pieces get fewer tiles.
+constexpr int kPieceCost = 8;
+
 struct schedule_t {
     std::vector<int32_t> cta_begin;
     std::vector<kvp_work> works;
@@ -203,12 +207,12 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, sche
                 u.n_all = (last / sh.group) / KVP_TILE_KEYS + 1 + n_prefix;
                 u.first_piece = u.n_pieces = 0;
                 units.push_back(u);
-                total += (int64_t)u.n_all * (u.mode ? 1 : 2);
+                total += (int64_t)u.n_all * (u.mode ? 1 : 2) + kPieceCost;
             }
     }
     int G = std::min(ctx->sm_count, kMaxCtas);
     if (ctx->split_target_ctas > 0) G = std::min(ctx->split_target_ctas, kMaxCtas);
-    if (total / G < 8) G = (int)std::max<int64_t>(1, total / 8);
+    if (total / G < 8 + kPieceCost) G = (int)std::max<int64_t>(1, total / (8 + kPieceCost));
     const bool no_split = ctx->force_splits == 1;               // cuts only between units
 
     // cut positions (unit, tile), non-decreasing
@@ -221,14 +225,14 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, sche
         for (int c = 1; c < G; ++c) {
             const int64_t target = total * c / G;
             while (u < units.size()) {
-                const int64_t cu = (int64_t)units[u].n_all * (units[u].mode ? 1 : 2);
+                const int64_t cu = (int64_t)units[u].n_all * (units[u].mode ? 1 : 2) + kPieceCost;
                 if (target < c_u + cu) break;
                 c_u += cu;
                 ++u;
             }
             if (u >= units.size()) break;
             const int w = units[u].mode ? 1 : 2;
-            int32_t t = (int32_t)((target - c_u + w / 2) / w);
+            int32_t t = (int32_t)std::max<int64_t>(0, (target - c_u - kPieceCost + w / 2) / w);
             if (no_split) t = (2 * t >= units[u].n_all) ? units[u].n_all : 0;
             if (t < 2) t = 0;
             if (units[u].n_all - t < 2) { cuts.push_back({(int32_t)u + 1, 0}); continue; }

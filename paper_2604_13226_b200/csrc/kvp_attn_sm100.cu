@@ -218,6 +218,15 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r)
         : "memory");
 }
 
+// tcgen05.ld fills its destination registers asynchronously, until tcgen05.wait::ld.  This empty
+// statement, placed after the wait, makes the compiler treat the 32 registers as written there, so that
+// no copy of them taken between the load and the wait can be used afterwards.
+#define KVP_RW8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), "+r"(r[o + 6]), "+r"(r[o + 7])
+__device__ __forceinline__ void landed32(uint32_t *r)
+{
+    asm volatile("" : KVP_RW8(r, 0), KVP_RW8(r, 8), KVP_RW8(r, 16), KVP_RW8(r, 24)::"memory");
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
@@ -335,7 +344,7 @@ __device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t
     const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
     auto lo_f = [](uint32_t u) { return __uint_as_float(u << 16); };
     auto hi_f = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
-#pragma unroll 2
+#pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         uint4 qa = __ldg(src + c), qb = __ldg(src + c + 8);
         uint32_t *a = reinterpret_cast<uint32_t *>(&qa);
@@ -398,23 +407,82 @@ __device__ __forceinline__ void chunk_mask(uint32_t *v, int lim)
     for (int i = 0; i < 32; ++i)
         if (i >= lim) v[i] = 0xff800000u;                  // -inf
 }
-// p = exp2(s*c2 - mc) for 32 scores; packed bf16 to 16 TMEM columns; returns their fp32 sum
-__device__ __forceinline__ float chunk_exp_store(const uint32_t *v, float c2, float mc, uint32_t p_addr)
+// ---- packed fp32 pairs (two lanes of the FMA pipe per instruction) --------------------------------------
+__device__ __forceinline__ uint64_t pair(float lo, float hi)
 {
-    uint32_t pk[16];
-    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpair(uint64_t r, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// p = exp2(s*c2 - mc) for 32 scores, packed as bf16 pairs into pk[16]; returns their fp32 sum.
+// (Evaluating part of the exponentials by a polynomial on the FMA pipe was measured and lost: the
+// extra issue slots cost more than the special-function unit saves.)
+__device__ __forceinline__ float chunk_exp(const uint32_t *v, float c2, float mc, uint32_t *pk)
+{
+    const uint64_t c2p = pair(c2, c2), nmc = pair(-mc, -mc);
+    uint64_t la = pair(0.f, 0.f), lb = pair(0.f, 0.f);
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        const float p0 = ex2(fmaf(__uint_as_float(v[i]), c2, -mc));
-        const float p1 = ex2(fmaf(__uint_as_float(v[i + 1]), c2, -mc));
-        const float p2 = ex2(fmaf(__uint_as_float(v[i + 2]), c2, -mc));
-        const float p3 = ex2(fmaf(__uint_as_float(v[i + 3]), c2, -mc));
-        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+    for (int i = 0; i < 32; i += 2) {
+        float x0, x1;
+        unpair(fma2(pair(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2p, nmc), x0, x1);
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        if (i & 2) lb = add2(lb, pair(p0, p1)); else la = add2(la, pair(p0, p1));
         pk[i >> 1] = pack_bf16(p0, p1);
-        pk[(i >> 1) + 1] = pack_bf16(p2, p3);
     }
-    tmem_st16(p_addr, pk);
-    return (l0 + l1) + (l2 + l3);
+    float s0, s1;
+    unpair(add2(la, lb), s0, s1);
+    return s0 + s1;
+}
+
+// Rare path of the softmax: the row's reference max moved up, so everything accumulated against the old
+// one shrinks by alpha = 2^(old - new): O in TMEM (when a P V product has been accumulated) and the P
+// chunks [0, n_chunks) of the current tile that were already written.  S of this step is complete, hence
+// so is the P V product of the previous step: O is quiet.
+__device__ __forceinline__ void rescale_row(uint32_t s_addr, uint32_t o_addr, float alpha, int n_chunks, bool with_o)
+{
+    uint32_t v[32];
+    if (with_o) {
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+            tmem_ld32(o_addr + ch * 32, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+            tmem_st32(o_addr + ch * 32, v);
+        }
+    }
+#pragma unroll 1
+    for (int ch = 0; ch < n_chunks; ++ch) {          // 16 columns of packed bf16 pairs per chunk
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : KVP_R8(v, 0), KVP_R8(v, 8)
+            : "r"(s_addr + ch * 16)
+            : "memory");
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            v[i] = pack_bf16(__uint_as_float(v[i] << 16) * alpha, __uint_as_float(v[i] & 0xffff0000u) * alpha);
+        tmem_st16(s_addr + ch * 16, v);
+    }
+    tc_wait_st();
 }
 
 __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, const int S, const int t)
@@ -453,53 +521,40 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
             const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);       // visible keys: [0, lim)
             uint32_t va[32], vb[32];
 
-            // pass 1: row max
-            float mx = -INFINITY;
-            tmem_ld32(s_addr, va);
-#pragma unroll 1
-            for (int ch = 0; ch < 4; ch += 2) {
-                tc_wait_ld();
-                tmem_ld32(s_addr + (ch + 1) * 32, vb);
-                if (!full) chunk_mask(va, lim - ch * 32);
-                mx = chunk_max(va, mx);
-                tc_wait_ld();
-                tmem_ld32(s_addr + ((ch + 2) & 3) * 32, va);          // last round: chunk 0 again, for pass 2
-                if (!full) chunk_mask(vb, lim - (ch + 1) * 32);
-                mx = chunk_max(vb, mx);
-            }
-            const float m_new = fmaxf(m_ref, mx);
-            if (k == 0) {
-                m_ref = m_new;
-            } else {
-                const bool need = (m_new - m_ref) * c2 > 8.0f;
+            // One pass over S: the exponentials use the reference max carried over from earlier tiles; each
+            // 32-column chunk's own max is checked first, and only if it exceeds the reference by more than
+            // 2^8 (first tile of a piece, or a rare jump) are l, O and the P chunks already written rescaled.
+            // The exponentials of a chunk are formed optimistically against the current reference while its
+            // max is reduced alongside; the check comes last, so the two dependency chains overlap.
+            auto process = [&](uint32_t *v, int ch) {
+                if (!full) chunk_mask(v, lim - ch * 32);
+                uint32_t pk[16];
+                const float cm = chunk_max(v, -INFINITY);
+                float ls = chunk_exp(v, c2, m_ref * c2, pk);
+                const bool need = (cm - m_ref) * c2 > 8.0f;
                 if (__any_sync(0xffffffffu, need)) {
-                    // S of this step is complete, hence so is the P V product of the previous step: O is quiet.
+                    const float m_new = need ? cm : m_ref;
                     const float alpha = need ? ex2((m_ref - m_new) * c2) : 1.f;
-                    if (need) m_ref = m_new;
+                    tc_wait_ld();                          // the other buffer's chunk may still be in flight
+                    landed32(v == va ? vb : va);
+                    rescale_row(s_addr, o_addr, alpha, ch, k > 0);
                     l *= alpha;
+                    m_ref = m_new;
+                    tmem_ld32(s_addr + ch * 32, v);             // this chunk's scores again (P so far lies below them)
                     tc_wait_ld();
-#pragma unroll 1
-                    for (int ch = 0; ch < 4; ++ch) {
-                        tmem_ld32(o_addr + ch * 32, vb);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
-                        tmem_st32(o_addr + ch * 32, vb);
-                    }
+                    landed32(v);
+                    if (!full) chunk_mask(v, lim - ch * 32);
+                    ls = chunk_exp(v, c2, m_ref * c2, pk);
                 }
-            }
-            // pass 2: p = exp2((s - m) c), written over S as packed bf16 (columns 0..63 of the S block)
-            const float mc = m_ref * c2;
+                tmem_st16(s_addr + ch * 16, pk);
+                l += ls;
+            };
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ch += 2) {
+            for (int ch = 0; ch < 4; ++ch) {
+                tmem_ld32(s_addr + ch * 32, va);
                 tc_wait_ld();
-                tmem_ld32(s_addr + (ch + 1) * 32, vb);
-                if (!full) chunk_mask(va, lim - ch * 32);
-                l += chunk_exp_store(va, c2, mc, s_addr + ch * 16);
-                tc_wait_ld();
-                if (ch == 0) tmem_ld32(s_addr + 64, va);
-                if (!full) chunk_mask(vb, lim - (ch + 1) * 32);
-                l += chunk_exp_store(vb, c2, mc, s_addr + (ch + 1) * 16);
+                landed32(va);
+                process(va, ch);
             }
             tc_wait_st();
             tc_fence_before();
@@ -543,7 +598,8 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
         }
         // un-normalised (partial slot) or normalised (output rows) O = w0 O_s (+ w1 O_1)
         uint4 *orow_bf = (direct && valid) ? reinterpret_cast<uint4 *>(p.out + (((long long)w.b * p.q_len + qi) * p.n_q + h) * 128) : nullptr;
-        uint4 *orow_f = direct ? nullptr : reinterpret_cast<uint4 *>(p.partial_o + ((long long)slot * KVP_TILE_ROWS + t) * 128);
+        // partial slot layout: [32 float4 columns][128 rows], so that a warp's store covers 512 contiguous bytes
+        uint4 *orow_f = direct ? nullptr : reinterpret_cast<uint4 *>(p.partial_o) + (long long)slot * (32 * KVP_TILE_ROWS) + t;
 #pragma unroll 1
         for (int ch = 0; ch < 4; ++ch) {
             uint32_t a[32];
@@ -570,7 +626,8 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
                 }
             } else if (orow_f != nullptr) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) orow_f[ch * 8 + i] = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+                for (int i = 0; i < 8; ++i)
+                    orow_f[(ch * 8 + i) * KVP_TILE_ROWS] = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
             }
         }
         if (direct) {
@@ -691,22 +748,60 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
     uint32_t ring_n = 0;
     bool ok = true;
 
+    // ---- S_s = Q_s K^T of step k of piece wq (whose loads start at ring position `base`) ----------------
+    auto issue_qk = [&](auto s_c, const Work &wq, uint32_t base, int k) {
+        constexpr int s = decltype(s_c)::value;
+        MmaStream &ms = st[s];
+        const int n_steps = s == 0 ? wq.steps0 : wq.steps1;
+        const bool shared_stage = (wq.mode == 0);                 // mode 0: both streams read the same K/V stage
+        if (k == 0) {
+            ms.prev_rope = 0;
+            ms.cur = get_tile(p, wq, stream_tile(wq, s, 0));
+            ms.nxt = n_steps > 1 ? get_tile(p, wq, stream_tile(wq, s, 1)) : ms.cur;
+        }
+        const Tile tl = ms.cur;
+        if (k == 0 || tl.rope != ms.prev_rope) {                  // first tile of a document: its own Q buffer
+            ms.qbuf = ms.nEpoch & 1;
+            ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
+            ++ms.nEpoch;
+        }
+        const int r = wq.mode ? 2 * k + s : k;
+        const uint32_t g = base + (uint32_t)load_seq(wq.mode, wq.n, r, 0);
+        const uint32_t stage = g % kStages, par = (g / kStages) & 1;
+        if (ok && !(shared_stage && s == 1)) ok = mbar_wait(c.bar(kKvFull + stage), par, c.abort_flag, p.status, 22);
+        ok = __all_sync(0xffffffffu, ok);                         // the lanes stay together
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
+        const uint32_t idesc = instr_desc(n16, 0);
+        const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
+        const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
+        const uint32_t d = c.tmem + kColS + s * 128;
+        mma_ss<0>(d, desc64(q_lo, kDescHi), desc64(k_lo, kDescHi), idesc);
+#pragma unroll
+        for (int kk = 1; kk < 8; ++kk) {                         // 16 columns per step: 32 bytes, second half 16 KB on
+            constexpr uint32_t kHalf16 = kHalfBytes >> 4;
+            const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
+            mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+        }
+        tc_commit(c.bar(kSFull + s));
+        if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
+        const bool last = (k + 1 == n_steps) || (ms.nxt.rope != tl.rope);
+        if (last) tc_commit(c.bar(kQFree + 2 * s + ms.qbuf));
+        ms.prev_rope = tl.rope;
+        ms.prev_keys = tl.n_keys;
+        ms.cur = ms.nxt;
+        if (k + 2 < n_steps) ms.nxt = get_tile(p, wq, stream_tile(wq, s, k + 2));
+    };
+
     for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
         const Work w = load_work(p, wi);
         const int steps[2] = {w.steps0, w.steps1};
         const int max_steps = max(w.steps0, w.steps1);
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            st[s].prev_rope = 0;
-            st[s].prev_keys = 0;
-            if (steps[s] > 0) st[s].cur = get_tile(p, w, stream_tile(w, s, 0));
-            if (steps[s] > 1) st[s].nxt = get_tile(p, w, stream_tile(w, s, 1));
-            else st[s].nxt = st[s].cur;
-        }
         auto block = [&](auto s_c, int k) {
             constexpr int s = decltype(s_c)::value;
             MmaStream &ms = st[s];
-            const bool shared_stage = (w.mode == 0);              // mode 0: both streams read the same K/V stage
+            const bool shared_stage = (w.mode == 0);
             if (k >= 1 && k <= steps[s]) {
                 // ---- O_s += P_s V of step k-1 -------------------------------------------------------
                 const int r = w.mode ? 2 * (k - 1) + s : k - 1;
@@ -717,7 +812,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 ++ms.nP;
                 if (ok && k == 1 && ms.nItems > 0)
                     ok = mbar_wait(c.bar(kOFree + s), (ms.nItems - 1) & 1, c.abort_flag, p.status, 26 + s);
-                ok = __all_sync(0xffffffffu, ok);                 // the lanes stay together
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t v_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, kHalfBytes);
@@ -738,42 +833,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                     ++ms.nItems;
                 }
             }
-            if (k < steps[s]) {
-                // ---- S_s = Q_s K^T of step k -------------------------------------------------------------
-                const Tile tl = ms.cur;
-                if (k == 0 || tl.rope != ms.prev_rope) {            // first tile of a document: its own Q buffer
-                    ms.qbuf = ms.nEpoch & 1;
-                    ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
-                    ++ms.nEpoch;
-                }
-                const int r = w.mode ? 2 * k + s : k;
-                const uint32_t g = ring_n + (uint32_t)load_seq(w.mode, w.n, r, 0);
-                const uint32_t stage = g % kStages, par = (g / kStages) & 1;
-                if (ok && !(shared_stage && s == 1)) ok = mbar_wait(c.bar(kKvFull + stage), par, c.abort_flag, p.status, 22);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
-                const uint32_t idesc = instr_desc(n16, 0);
-                const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
-                const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
-                const uint32_t d = c.tmem + kColS + s * 128;
-                mma_ss<0>(d, desc64(q_lo, kDescHi), desc64(k_lo, kDescHi), idesc);
-#pragma unroll
-                for (int kk = 1; kk < 8; ++kk) {                 // 16 columns per step: 32 bytes, second half 16 KB on
-                    constexpr uint32_t kHalf16 = kHalfBytes >> 4;
-                    const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
-                    mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
-                }
-                tc_commit(c.bar(kSFull + s));
-                if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
-                const bool last = (k + 1 == steps[s]) || (ms.nxt.rope != tl.rope);
-                if (last) tc_commit(c.bar(kQFree + 2 * s + ms.qbuf));
-                ms.prev_rope = tl.rope;
-                ms.prev_keys = tl.n_keys;
-                ms.cur = ms.nxt;
-                if (k + 2 < steps[s]) ms.nxt = get_tile(p, w, stream_tile(w, s, k + 2));
-            }
+            if (k < steps[s]) issue_qk(s_c, w, ring_n, k);
         };
         for (int k = 0; k <= max_steps && ok; ++k) {
             block(std::integral_constant<int, 0>{}, k);
@@ -864,42 +924,65 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
 }
 
 // ---- merge of the partial slots of split units ------------------------------------------------------------
-// Partials hold, per (slot, row): un-normalised O (fp32), the running max m of the raw scores and the
-// sum l of exp2((s - m) * c).  Block = 8 rows x 32 float4 columns; grid (merge item, 16).
+// Partials hold, per (slot, row): un-normalised O (fp32, stored [32 float4 columns][128 rows]), the
+// running max m of the raw scores and the sum l of exp2((s - m) * c).  Block = 32 rows of one merge
+// item; lanes run along rows while reading (coalesced), the result is turned through shared memory so
+// that the bf16 output rows are written 256 contiguous bytes at a time.  Grid (merge item, 4).
 __global__ void __launch_bounds__(256)
 merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q, int group, float scale,
                   const float *__restrict__ part_o, const float2 *__restrict__ part_ml,
                   __nv_bfloat16 *__restrict__ out, float *__restrict__ lse)
 {
+    __shared__ uint2 tile[32][33];
     const kvp_merge_item mi = merges[blockIdx.x];
-    const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
-    const int c4 = threadIdx.x & 31;
-    const int r = mi.row_base + row;
-    if (r >= group * q_len) return;
+    const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5;
+    const int row = blockIdx.y * 32 + lane;                     // row of the 128-row query tile
+    const int n_rows = group * q_len;
     const float c2 = scale * 1.4426950408889634f;
+    const float4 *po = reinterpret_cast<const float4 *>(part_o);
     float M = -INFINITY;
     for (int s = 0; s < mi.n_slots; ++s) {
         const float2 ml = part_ml[(long long)(mi.slot0 + s) * KVP_TILE_ROWS + row];
         if (ml.y > 0.f) M = fmaxf(M, ml.x);
     }
     float L = 0.f;
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < mi.n_slots; ++s) {
-        const long long base = (long long)(mi.slot0 + s) * KVP_TILE_ROWS + row;
-        const float2 ml = part_ml[base];
-        if (!(ml.y > 0.f)) continue;                    // an empty partial: nothing was visible to this row
+        const long long slot = mi.slot0 + s;
+        const float2 ml = part_ml[slot * KVP_TILE_ROWS + row];
+        if (!(ml.y > 0.f)) continue;                            // an empty partial: nothing was visible to this row
         const float w = exp2f((ml.x - M) * c2);
         L += w * ml.y;
-        const float4 a = reinterpret_cast<const float4 *>(part_o + base * 128)[c4];
-        o.x += w * a.x; o.y += w * a.y; o.z += w * a.z; o.w += w * a.w;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float4 a = po[(slot * 32 + wv + 8 * j) * KVP_TILE_ROWS + row];
+            o[j].x += w * a.x; o[j].y += w * a.y; o[j].z += w * a.z; o[j].w += w * a.w;
+        }
     }
-    const float inv = 1.f / L;
-    const int i = r / group, h = mi.hk * group + r % group;
-    uint2 u;
-    u.x = pack_bf16(o.x * inv, o.y * inv);
-    u.y = pack_bf16(o.z * inv, o.w * inv);
-    reinterpret_cast<uint2 *>(out + (((long long)mi.b * q_len + i) * n_q + h) * 128)[c4] = u;
-    if (c4 == 0 && lse != nullptr) lse[((long long)mi.b * n_q + h) * q_len + i] = M * scale + logf(L);
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint2 u;
+        u.x = pack_bf16(o[j].x * inv, o[j].y * inv);
+        u.y = pack_bf16(o[j].z * inv, o[j].w * inv);
+        tile[lane][wv + 8 * j] = u;
+    }
+    const int r = mi.row_base + row;
+    if (wv == 0 && r < n_rows && lse != nullptr)
+        lse[((long long)mi.b * n_q + mi.hk * group + r % group) * q_len + r / group] = M * scale + logf(L);
+    __syncthreads();
+    // 8 threads per output row, 32 bytes each
+    const int orow = threadIdx.x >> 3, j8 = threadIdx.x & 7;
+    const int r2 = mi.row_base + blockIdx.y * 32 + orow;
+    if (r2 < n_rows) {
+        const int i = r2 / group, h = mi.hk * group + r2 % group;
+        uint4 *dst = reinterpret_cast<uint4 *>(out + (((long long)mi.b * q_len + i) * n_q + h) * 128) + 2 * j8;
+        const uint2 a0 = tile[orow][4 * j8], a1 = tile[orow][4 * j8 + 1], a2 = tile[orow][4 * j8 + 2], a3 = tile[orow][4 * j8 + 3];
+        dst[0] = make_uint4(a0.x, a0.y, a1.x, a1.y);
+        dst[1] = make_uint4(a2.x, a2.y, a3.x, a3.y);
+    }
 }
 
 }  // namespace
@@ -940,7 +1023,7 @@ cudaError_t kvp_launch_merge_list(const kvp_shape &sh, int32_t q_len, int32_t n_
                                   cudaStream_t st)
 {
     if (n_merges <= 0) return cudaSuccess;
-    merge_list_kernel<<<dim3(n_merges, KVP_TILE_ROWS / 8), 256, 0, st>>>(merges, q_len, sh.n_q_heads, sh.group, sh.scale,
+    merge_list_kernel<<<dim3(n_merges, KVP_TILE_ROWS / 32), 256, 0, st>>>(merges, q_len, sh.n_q_heads, sh.group, sh.scale,
                                                                         partial_o, partial_ml, (__nv_bfloat16 *)out, lse);
     return cudaGetLastError();
 }
