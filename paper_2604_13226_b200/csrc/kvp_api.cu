@@ -212,33 +212,49 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, sche
     }
     int G = std::min(ctx->sm_count, kMaxCtas);
     if (ctx->split_target_ctas > 0) G = std::min(ctx->split_target_ctas, kMaxCtas);
-    if (total / G < 8 + kPieceCost) G = (int)std::max<int64_t>(1, total / (8 + kPieceCost));
     const bool no_split = ctx->force_splits == 1;               // cuts only between units
 
-    // cut positions (unit, tile), non-decreasing
+    // Cut positions (unit, tile), non-decreasing.  CTAs are filled one after the other up to a budget;
+    // every piece pays kPieceCost on top of its tiles, a piece is at least two tiles long (or the whole
+    // unit), and without splitting a unit goes to the CTA that holds its larger part.  The smallest
+    // budget that needs no more than G CTAs is found by bisection.
     struct cut_t { int32_t u, t; };
     std::vector<cut_t> cuts;
-    cuts.push_back({0, 0});
-    {
+    auto fill = [&](int64_t budget, std::vector<cut_t> *rec) -> int {
+        int used = 0;
         size_t u = 0;
-        int64_t c_u = 0;                                        // cost before unit u
-        for (int c = 1; c < G; ++c) {
-            const int64_t target = total * c / G;
+        int32_t t = 0;
+        while (u < units.size()) {
+            ++used;
+            if (rec) rec->push_back({(int32_t)u, t});
+            int64_t cost = 0;
             while (u < units.size()) {
-                const int64_t cu = (int64_t)units[u].n_all * (units[u].mode ? 1 : 2) + kPieceCost;
-                if (target < c_u + cu) break;
-                c_u += cu;
-                ++u;
+                const int w = units[u].mode ? 1 : 2;
+                const int32_t left = units[u].n_all - t;
+                const int64_t room = budget - cost - kPieceCost;
+                int32_t take = (int32_t)std::min<int64_t>(left, room > 0 ? (room + w - 1) / w : 0);
+                if (no_split) take = (t == 0 && (2 * take >= left || cost == 0)) ? left : 0;
+                if (left - take < 2) take = left;                 // do not leave a sliver behind
+                if (take < 2 && take < left) take = 0;
+                if (take == 0) {
+                    if (cost > 0) break;                          // start the piece in the next CTA
+                    take = no_split ? left : std::min<int32_t>(left, 2);
+                    if (left - take < 2) take = left;
+                }
+                cost += kPieceCost + (int64_t)take * w;
+                t += take;
+                if (t == units[u].n_all) { ++u; t = 0; }
+                if (cost >= budget) break;
             }
-            if (u >= units.size()) break;
-            const int w = units[u].mode ? 1 : 2;
-            int32_t t = (int32_t)std::max<int64_t>(0, (target - c_u - kPieceCost + w / 2) / w);
-            if (no_split) t = (2 * t >= units[u].n_all) ? units[u].n_all : 0;
-            if (t < 2) t = 0;
-            if (units[u].n_all - t < 2) { cuts.push_back({(int32_t)u + 1, 0}); continue; }
-            cuts.push_back({(int32_t)u, t});
         }
+        return used;
+    };
+    int64_t lo_b = std::max<int64_t>(total / G, 8 + kPieceCost), hi_b = total + kPieceCost;
+    while (lo_b < hi_b) {
+        const int64_t mid = (lo_b + hi_b) / 2;
+        if (fill(mid, nullptr) <= G) hi_b = mid; else lo_b = mid + 1;
     }
+    fill(lo_b, &cuts);
     cuts.push_back({(int32_t)units.size(), 0});
 
     std::vector<kvp_work> &works = out.works;
