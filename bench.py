@@ -10,7 +10,8 @@ prints ONE JSON line.  ``value`` = query tokens/s of the whole job (batch * q_le
 full layer stack per step), inputs resident in HBM.  ``e2e`` = the same with the step's Q/K_new/V_new
 coming from pinned host buffers and the outputs read back, copies inside the timed region.
 ``roofline`` is for the dominant kernel (the tcgen05 attention kernel), its duration measured live
-with CUDA events on the launching stream.  ``cpu_baseline`` is the fp64 oracle on the host cores on a
+with CUDA events on the launching stream.  ``extra_points`` add the memory-bound short-query shape, the
+gather kernel in materialise mode and a decode step (one token per request).  ``cpu_baseline`` is the fp64 oracle on the host cores on a
 bounded sample.  ``--impl reference`` times that oracle as the reference arm.
 
 Workloads (seeded, synthetic, shaped like the paper's Llama-3.1-8B / Qwen2.5-7B RAG requests):
@@ -421,6 +422,8 @@ def main():
             try:
                 extras["hbm_bound_point"] = measure_point("config5:64:16:1", args.seed, 10, False, peaks, local_rank)
                 extras["gather_materialise_point"] = measure_point("config5:16:64:1", args.seed, 10, True, peaks, local_rank)
+                # the step after the prefill: one new token per request over 16 x 33,280-token composed caches
+                extras["decode_point"] = measure_point("config5:16:1:16", args.seed, 10, False, peaks, local_rank)
             except Exception as ex:                                   # extras never invalidate the main line
                 extras["error"] = repr(ex)
             line["extra_points"] = extras

@@ -54,7 +54,8 @@ enum {
 /* kvp_query_prefill flags */
 enum {
     KVP_ROPE_QUERY = 1u,      /* q and k_new are raw: rotate them at positions prefix_len[b] + i        */
-    KVP_FORCE_SIMPLE = 2u     /* use the plain fp32 CUDA-core kernel (cross-check path, any dtype)      */
+    KVP_FORCE_SIMPLE = 2u,    /* use the plain fp32 CUDA-core kernel (cross-check path, any dtype)      */
+    KVP_CONTINUE = 4u         /* the q_len tokens follow the rows this layer's earlier calls appended   */
 };
 
 typedef struct kvp_ctx kvp_ctx;
@@ -152,7 +153,12 @@ KVP_API int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_of
  *   out    device [batch][q_len][n_q_heads][head_dim]
  *   lse    device float [batch][n_q_heads][q_len] or NULL: natural-log sum of exp(scaled scores)
  * By default q and k_new are already rotated for positions prefix_len[b] + i; KVP_ROPE_QUERY makes
- * the library rotate them.  Errors: INVALID, NOT_FOUND, CAPACITY (q_len > max_query_tokens),
+ * the library rotate them.
+ * KVP_CONTINUE (the step after the prefill - decoding with q_len = 1 - or a prefill fed in chunks): the
+ * rows appended by the earlier calls for this layer since kvp_assemble stay; with n of them, token i of
+ * this call sits at position prefix_len[b] + n + i, attends to the prefix, to those n rows and to this
+ * call's tokens <= i, and is appended behind them.  n + q_len may not exceed max_query_tokens.  Without
+ * the flag a call starts again at prefix_len[b].  Errors: INVALID, NOT_FOUND, CAPACITY (q_len > max_query_tokens),
  * STATE (host-only context), UNSUPPORTED, CUDA.  Device-side wait timeouts are reported through
  * kvp_status_word after the stream has been synchronised.
  */

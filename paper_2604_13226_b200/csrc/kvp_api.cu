@@ -189,7 +189,7 @@ struct schedule_t {
     int32_t n_ctas = 0, n_slots = 0, max_pieces = 1;
 };
 
-int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, schedule_t &out)
+int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, int q_pos0, schedule_t &out)
 {
     const kvp_shape &sh = ctx->shape;
     struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces; };
@@ -204,7 +204,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, sche
                 u.b = b; u.hk = hk; u.row_base = row_base;
                 u.mode = (n_rows - row_base <= KVP_TILE_ROWS) ? 1 : 0;
                 const int last = std::min(n_rows - 1, row_base + (u.mode ? 1 : 2) * KVP_TILE_ROWS - 1);
-                u.n_all = (last / sh.group) / KVP_TILE_KEYS + 1 + n_prefix;
+                u.n_all = (q_pos0 + last / sh.group) / KVP_TILE_KEYS + 1 + n_prefix;
                 u.first_piece = u.n_pieces = 0;
                 units.push_back(u);
                 total += (int64_t)u.n_all * (u.mode ? 1 : 2) + kPieceCost;
@@ -312,10 +312,10 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, sche
     return KVP_OK;
 }
 
-int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len, cudaStream_t st)
+int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len, int q_pos0, cudaStream_t st)
 {
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, as, q_len, sc);
+    const int32_t rc = plan_schedule(ctx, as, q_len, q_pos0, sc);
     if (rc != KVP_OK) return rc;
     const std::vector<int32_t> &cta_begin = sc.cta_begin;
     const std::vector<kvp_work> &works = sc.works;
@@ -336,6 +336,7 @@ int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len,
                                       sizeof(kvp_merge_item) * merges.size(), cudaMemcpyHostToDevice, st));
     KVP_CUDA(ctx, cudaEventRecord(ctx->sched_event[slot], st));
     as.sched_q_len = q_len;
+    as.sched_q_pos0 = q_pos0;
     as.sched_ctas = n_ctas;
     as.sched_works = (int32_t)works.size();
     as.sched_merges = (int32_t)merges.size();
@@ -749,41 +750,47 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "query_prefill: unknown assembly %d", assembly_id);
     if (!q || !k_new || !v_new || !out || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
         return fail(ctx, KVP_ERR_INVALID, "query_prefill: bad arguments");
-    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE | KVP_CONTINUE)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
     if (q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: q_len > max_query_tokens");
     kvp_assembly_host &as = ctx->slots[slot];
     const kvp_shape &sh = ctx->shape;
     cudaStream_t st = (cudaStream_t)stream;
+    if ((int)as.appended.size() != ctx->cfg.n_layers) as.appended.assign(ctx->cfg.n_layers, 0);
+    const int q_pos0 = (flags & KVP_CONTINUE) ? as.appended[layer] : 0;
+    if (q_pos0 + q_len > ctx->cfg.max_query_tokens)
+        return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: %d rows appended + q_len %d > max_query_tokens", q_pos0, q_len);
     KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     const kvp_plan_dev plan = plan_dev(ctx, slot);
     const int rope_query = (flags & KVP_ROPE_QUERY) ? 1 : 0;
     const double *inv_freq_dev = reinterpret_cast<const double *>((char *)ctx->cfg.workspace + 256);
 
     int launches = 0;
-    KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
+    KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q_pos0, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
                                     layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
     ++launches;
     const void *q_used = rope_query ? (const void *)ctx->q_scratch : q;
     as.last_q_len = q_len;
+    as.appended[layer] = q_pos0 + q_len;
 
     const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
     int32_t ctas = 0, splits = 1;
     if (!fast) {
         KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
-        KVP_CUDA(ctx, kvp_launch_attn_simple(sh, plan, as.batch, q_len, layer, q_used, ctx->pool_k, ctx->pool_v,
+        KVP_CUDA(ctx, kvp_launch_attn_simple(sh, plan, as.batch, q_len, q_pos0, layer, q_used, ctx->pool_k, ctx->pool_v,
                                              ctx->slot_k[slot], ctx->slot_v[slot], out, lse, &ctas, st));
         KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
         ctx->last_kind = 0;
     } else if (ctx->kernel_variant == 0) {
-        if (as.sched_q_len != q_len || as.sched_ctas == 0) {
-            const int32_t rc = build_schedule(ctx, as, slot, q_len, st);
+        if (as.sched_q_len != q_len || as.sched_q_pos0 != q_pos0 || as.sched_ctas == 0) {
+            const int32_t rc = build_schedule(ctx, as, slot, q_len, q_pos0, st);
             if (rc != KVP_OK) return rc;
         }
         const char *sd = ctx->slot_sched_dev[slot];
         kvp_attn2_args a;
         a.plan = plan;
         a.q_len = q_len;
+        a.q_pos0 = q_pos0;
         a.layer = layer;
         a.n_ctas = as.sched_ctas;
         a.cta_begin = reinterpret_cast<const int32_t *>(sd);
@@ -808,6 +815,7 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         splits = as.sched_slots;
         ctx->last_kind = 1;
     } else {
+        if (q_pos0 > 0) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: the single-tile kernel variant has no KVP_CONTINUE");
         const int n_mtiles = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
         const int units = as.batch * sh.n_kv_heads * n_mtiles;
         int min_tiles = INT32_MAX;
@@ -883,7 +891,7 @@ int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, in
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_schedule: unknown assembly %d", assembly_id);
     if (q_len <= 0 || q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_INVALID, "export_schedule: bad q_len");
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], q_len, sc);
+    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], q_len, 0, sc);
     if (rc != KVP_OK) return rc;
     counts[0] = sc.n_ctas;
     counts[1] = (int32_t)sc.works.size();

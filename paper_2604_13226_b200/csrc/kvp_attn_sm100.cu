@@ -56,7 +56,7 @@ static_assert(8 * kNumBars + 8 <= 256, "barrier block");
 
 struct Params {
     kvp_plan_dev plan;
-    int q_len, layer, n_q, n_kv, group, pairing;
+    int q_len, q_pos0, layer, n_q, n_kv, group, pairing;      // q_pos0: tail rows appended by earlier calls
     float scale, scale_log2;
     const int32_t *cta_begin;
     const kvp_work *works;
@@ -281,7 +281,7 @@ __device__ __forceinline__ Work load_work(const Params &p, int wi)
     w.tail_row0 = ib.y;
     const int n_rows = p.group * p.q_len;
     const int last = min(n_rows - 1, w.row_base + (w.mode ? KVP_TILE_ROWS : 2 * KVP_TILE_ROWS) - 1);
-    w.n_tail = (last / p.group) / KVP_TILE_KEYS + 1;
+    w.n_tail = (p.q_pos0 + last / p.group) / KVP_TILE_KEYS + 1;
     w.plane = p.layer * p.n_kv + w.hk;
     w.steps0 = w.mode ? (w.n + 1) >> 1 : w.n;
     w.steps1 = w.mode ? w.n >> 1 : w.n;
@@ -298,7 +298,7 @@ __device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
     Tile t;
     if (j < w.n_tail) {
         t.row0 = w.tail_row0 + j * KVP_TILE_KEYS;
-        t.n_keys = min(KVP_TILE_KEYS, p.q_len - j * KVP_TILE_KEYS);
+        t.n_keys = min(KVP_TILE_KEYS, p.q_pos0 + p.q_len - j * KVP_TILE_KEYS);
         t.src = 1;
         t.rope = 0;
         t.qoff = j * KVP_TILE_KEYS;
@@ -518,7 +518,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
             tc_fence_after();
 
             const bool full = (tl.n_keys == KVP_TILE_KEYS) && (tl.qoff < 0);
-            const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, qi - tl.qoff + 1);       // visible keys: [0, lim)
+            const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, p.q_pos0 + qi - tl.qoff + 1);       // visible keys: [0, lim)
             uint32_t va[32], vb[32];
 
             // One pass over S: the exponentials use the reference max carried over from earlier tiles; each
@@ -999,6 +999,7 @@ cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, 
     Params p;
     p.plan = a.plan;
     p.q_len = a.q_len;
+    p.q_pos0 = a.q_pos0;
     p.layer = a.layer;
     p.n_q = sh.n_q_heads;
     p.n_kv = sh.n_kv_heads;

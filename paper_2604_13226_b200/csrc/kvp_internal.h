@@ -108,7 +108,9 @@ struct kvp_assembly_host {
     std::vector<kvp_tile> tiles;
     int32_t n_chunks = 0, n_rope = 0;
     int32_t last_q_len = 0;
-    // work list of the two-stream kernel, built for sched_q_len query tokens (0 = none yet)
+    std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
+    // work list of the two-stream kernel, built for sched_q_len query tokens at offset sched_q_pos0 (0 = none yet)
+    int32_t sched_q_pos0 = 0;
     int32_t sched_q_len = 0, sched_ctas = 0, sched_works = 0, sched_merges = 0, sched_slots = 0;
 };
 
@@ -166,7 +168,7 @@ cudaError_t kvp_launch_store_rows(const kvp_shape &sh, const void *src, char *ds
 cudaError_t kvp_launch_gather(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t n_chunks,
                               const char *pool_k, const char *pool_v, char *ws_k, char *ws_v, cudaStream_t st);
 cudaError_t kvp_launch_append(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
-                              const void *q, const void *k_new, const void *v_new, char *ws_k, char *ws_v,
+                              int32_t q_pos0, const void *q, const void *k_new, const void *v_new, char *ws_k, char *ws_v,
                               int32_t layer, int32_t rope_query, const double *inv_freq_dev, void *q_rot,
                               cudaStream_t st);
 cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t b, int32_t layer,
@@ -174,7 +176,7 @@ cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int
                               const char *ws_k, const char *ws_v, void *k_out, void *v_out, int32_t k_as_f32,
                               cudaStream_t st);
 cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
-                                   int32_t layer, const void *q, const char *pool_k, const char *pool_v,
+                                   int32_t q_pos0, int32_t layer, const void *q, const char *pool_k, const char *pool_v,
                                    const char *ws_k, const char *ws_v, void *out, float *lse, int32_t *ctas,
                                    cudaStream_t st);
 
@@ -198,7 +200,7 @@ cudaError_t kvp_launch_attn_sm100_single(const kvp_shape &sh, const kvp_attn_sm1
 
 struct kvp_attn2_args {
     kvp_plan_dev plan;
-    int32_t q_len, layer, n_ctas;
+    int32_t q_len, q_pos0, layer, n_ctas;
     const int32_t *cta_begin;      // [n_ctas + 1] ranges into works
     const kvp_work *works;
     const void *q;

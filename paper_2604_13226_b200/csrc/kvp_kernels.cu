@@ -117,10 +117,10 @@ __global__ void gather_kernel(kvp_plan_dev plan, const char *__restrict__ pool_k
 }
 
 // ---- append: the query chunk's own K/V rows go behind the prefix (Section 3.2 step 4) --------------
-// grid (batch*q_len); with rope_query the raw k_new and q are first rotated to positions
-// prefix_len + i, angles formed in double precision.
+// grid (batch*q_len); the rows go behind the q_pos0 rows appended earlier; with rope_query the raw
+// k_new and q are first rotated to positions prefix_len + q_pos0 + i, angles formed in double precision.
 template <typename T>
-__global__ void append_kernel(kvp_plan_dev plan, int q_len, const T *__restrict__ q, const T *__restrict__ k_new,
+__global__ void append_kernel(kvp_plan_dev plan, int q_len, int q_pos0, const T *__restrict__ q, const T *__restrict__ k_new,
                               const T *__restrict__ v_new, char *__restrict__ ws_k, char *__restrict__ ws_v,
                               int64_t ws_rows, int layer, int n_q, int n_kv, int d, int pairing, int rope_query,
                               const double *__restrict__ inv_freq, T *__restrict__ q_rot)
@@ -132,7 +132,7 @@ __global__ void append_kernel(kvp_plan_dev plan, int q_len, const T *__restrict_
     if (rope_query) {
         for (int p = threadIdx.x; p < half; p += blockDim.x) {
             double s, c;
-            sincos((double)(it.prefix_len + i) * inv_freq[p], &s, &c);
+            sincos((double)(it.prefix_len + q_pos0 + i) * inv_freq[p], &s, &c);
             cs[p] = make_float2((float)c, (float)s);
         }
         __syncthreads();
@@ -144,7 +144,7 @@ __global__ void append_kernel(kvp_plan_dev plan, int q_len, const T *__restrict_
         const int ia = pairing ? 2 * p : p, ib = pairing ? 2 * p + 1 : p + half;
         const T *ks = k_new + (tok * n_kv + hk) * d;
         const T *vs = v_new + (tok * n_kv + hk) * d;
-        const int64_t drow = ((int64_t)(layer * n_kv + hk)) * ws_rows + it.tail_row0 + i;
+        const int64_t drow = ((int64_t)(layer * n_kv + hk)) * ws_rows + it.tail_row0 + q_pos0 + i;
         T *kd = reinterpret_cast<T *>(ws_k) + drow * d;
         T *vd = reinterpret_cast<T *>(ws_v) + drow * d;
         float a = Elem<T>::to_f32(ks[ia]), bb = Elem<T>::to_f32(ks[ib]);
@@ -241,7 +241,7 @@ __global__ void export_kernel(kvp_plan_dev plan, int b, int layer, int prefix_le
 // Keys still carrying an offset are rotated here as Eq. 1 states it (on K, in fp32).
 template <typename T, int D>
 __global__ void __launch_bounds__(128)
-attn_simple_kernel(kvp_plan_dev plan, int q_len, int layer, const T *__restrict__ q, const char *__restrict__ pool_k,
+attn_simple_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T *__restrict__ q, const char *__restrict__ pool_k,
                    const char *__restrict__ pool_v, const char *__restrict__ ws_k, const char *__restrict__ ws_v,
                    int64_t pool_rows, int64_t ws_rows, int n_q, int n_kv, int group, int pairing, float scale,
                    T *__restrict__ out, float *__restrict__ lse)
@@ -271,7 +271,7 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int layer, const T *__restrict_
 
     const int last_row = min(n_rows - 1, blockIdx.x * RB + RB - 1);
     const int i_max = last_row / group;
-    const int n_tail = i_max / KVP_TILE_KEYS + 1;
+    const int n_tail = (q_pos0 + i_max) / KVP_TILE_KEYS + 1;      // tail keys: rows appended earlier, then this call's
     const int n_tiles = n_tail + (it.tile_end - it.tile_begin);
 
     float m = -1e30f, l = 0.f;
@@ -284,7 +284,7 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int layer, const T *__restrict_
         int qoff = -1;
         if (tt < n_tail) {
             tl.row0 = it.tail_row0 + tt * KVP_TILE_KEYS;
-            tl.n_keys = (int16_t)min(KVP_TILE_KEYS, q_len - tt * KVP_TILE_KEYS);
+            tl.n_keys = (int16_t)min(KVP_TILE_KEYS, q_pos0 + q_len - tt * KVP_TILE_KEYS);
             tl.src = 1;
             tl.rope = 0;
             qoff = tt * KVP_TILE_KEYS;
@@ -327,7 +327,7 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int layer, const T *__restrict_
                 float a = 0.f;
 #pragma unroll 8
                 for (int c = 0; c < D; ++c) a += Qs[row][c] * Ks[kk][c];
-                const bool vis = kk < nk && (qoff < 0 || qoff + k0 + kk <= i);
+                const bool vis = kk < nk && (qoff < 0 || qoff + k0 + kk <= q_pos0 + i);
                 s[u] = vis ? a * scale : -INFINITY;
                 mx = fmaxf(mx, s[u]);
             }
@@ -434,18 +434,18 @@ cudaError_t kvp_launch_gather(const kvp_shape &sh, const kvp_plan_dev &plan, int
 }
 
 cudaError_t kvp_launch_append(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
-                              const void *q, const void *k_new, const void *v_new, char *ws_k, char *ws_v,
+                              int32_t q_pos0, const void *q, const void *k_new, const void *v_new, char *ws_k, char *ws_v,
                               int32_t layer, int32_t rope_query, const double *inv_freq_dev, void *q_rot,
                               cudaStream_t st)
 {
     const int grid = batch * q_len;
     if (sh.dtype == KVP_DTYPE_BF16)
         append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-            plan, q_len, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k_new, (const __nv_bfloat16 *)v_new, ws_k,
+            plan, q_len, q_pos0, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k_new, (const __nv_bfloat16 *)v_new, ws_k,
             ws_v, sh.ws_rows, layer, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.pairing, rope_query, inv_freq_dev,
             (__nv_bfloat16 *)q_rot);
     else
-        append_kernel<float><<<grid, 256, 0, st>>>(plan, q_len, (const float *)q, (const float *)k_new,
+        append_kernel<float><<<grid, 256, 0, st>>>(plan, q_len, q_pos0, (const float *)q, (const float *)k_new,
                                                    (const float *)v_new, ws_k, ws_v, sh.ws_rows, layer, sh.n_q_heads,
                                                    sh.n_kv_heads, sh.head_dim, sh.pairing, rope_query, inv_freq_dev,
                                                    (float *)q_rot);
@@ -472,14 +472,14 @@ cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int
 }
 
 cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
-                                   int32_t layer, const void *q, const char *pool_k, const char *pool_v,
+                                   int32_t q_pos0, int32_t layer, const void *q, const char *pool_k, const char *pool_v,
                                    const char *ws_k, const char *ws_v, void *out, float *lse, int32_t *ctas,
                                    cudaStream_t st)
 {
     const dim3 grid((sh.group * q_len + 15) / 16, sh.n_kv_heads, batch);
     if (ctas) *ctas = (int32_t)(grid.x * grid.y * grid.z);
 #define KVP_SIMPLE(T, D)                                                                                             \
-    attn_simple_kernel<T, D><<<grid, 128, 0, st>>>(plan, q_len, layer, (const T *)q, pool_k, pool_v, ws_k, ws_v,     \
+    attn_simple_kernel<T, D><<<grid, 128, 0, st>>>(plan, q_len, q_pos0, layer, (const T *)q, pool_k, pool_v, ws_k, ws_v,     \
                                                    sh.pool_rows, sh.ws_rows, sh.n_q_heads, sh.n_kv_heads, sh.group,  \
                                                    sh.pairing, sh.scale, (T *)out, lse)
     if (sh.dtype == KVP_DTYPE_BF16) {
