@@ -87,6 +87,8 @@ typedef struct kvp_config {
                                    (adapter tokens + max_query_tokens), or with KVP_MATERIALIZE of
                                    (prefix tokens + max_query_tokens)                                  */
     int32_t max_assemblies;     /* assemblies alive at once (ring; ids older than this are dropped)   */
+    int32_t max_compressed;     /* compressed packets one assembly may use (0: none; sizes the per-layer
+                                   tile lists and the table of kept counts)                            */
 } kvp_config;
 
 /* Bytes of pool one token occupies (K and V, all layers and kv heads).  0 if cfg is invalid. */
@@ -115,6 +117,25 @@ KVP_API int32_t kvp_destroy(kvp_ctx *ctx);
  */
 KVP_API int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens,
                             int32_t cache_pos0, void *stream, int32_t *packet_id);
+
+/*
+ * Register one compressed packet: a document cache after unstructured KV pruning (Section 4.3,
+ * "Compatibility with KV Compression": compressors keep a different token subset per layer - and, for
+ * many of them, per head - and the method composes such caches as opaque units).  Layer l, kv head h keeps
+ * kept[l * n_kv_heads + h] of the document's n_tokens keys and values (>= 1 each); which tokens is the
+ * compressor's business: every key carries the rotation of the position it was cached at and the packet
+ * keeps those positions, so it still takes one offset Delta, and its extent in a request stays n_tokens
+ * positions (the next segment starts n_tokens further on).
+ *   k, v   device; for (l, h) in that order, kept[l][h] rows of head_dim elements, the runs back to back
+ *   kept   host [n_layers][n_kv_heads]
+ * The packet occupies max(kept) pool rows.  Needs cfg.max_compressed > 0.  Assemblies that use a
+ * compressed packet cannot be materialised (KVP_MATERIALIZE) or exported with kvp_export_cache, and run
+ * on the two-stream tcgen05 kernel or the CUDA-core kernel only: those return KVP_ERR_UNSUPPORTED.
+ * Errors: INVALID, CAPACITY (max_packets, pool), STATE (max_compressed == 0), CUDA.
+ */
+KVP_API int32_t kvp_register_packet_compressed(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens,
+                                               int32_t cache_pos0, const int32_t *kept, void *stream,
+                                               int32_t *packet_id);
 
 /*
  * Register one adapter: K/V of N_h header and N_t trailer soft tokens (Section 3.1, phi = {H, T}),

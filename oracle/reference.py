@@ -120,11 +120,17 @@ class Store:
         self.rows = 0
         self.packets: List[Tuple[_Segment, Callable]] = []
         self.adapters: List[Tuple[_Segment, _Segment, Callable]] = []
+        self.kept: dict = {}       # packet id -> kept[layer][kv_head] token indices (compressed packets only)
 
-    def register_packet(self, n_tokens: int, cache_pos0: int, loader: Callable) -> int:
+    def register_packet(self, n_tokens: int, cache_pos0: int, loader: Callable, kept=None) -> int:
+        """``kept`` marks a compressed packet (Section 4.3): after unstructured pruning, layer l / kv head h
+        of its cache holds only the tokens ``kept[l][h]``; the loader still returns the full document and
+        the packet still spans n_tokens positions (pruned tokens leave their positions unoccupied)."""
         seg = _Segment(self.rows, int(n_tokens), int(cache_pos0))
         self.rows += int(n_tokens)
         self.packets.append((seg, loader))
+        if kept is not None:
+            self.kept[len(self.packets) - 1] = kept
         return len(self.packets) - 1
 
     def register_adapter(self, n_header: int, header_pos0: int, n_trailer: int, trailer_pos0: int,
@@ -249,5 +255,43 @@ def query_prefill(store: Store, plan: Plan, layer: int, q, k_new, v_new, inv_f: 
     V = np.concatenate([Vp, Vn], axis=0)
     if scale is None:
         scale = 1.0 / np.sqrt(np.float64(d))
-    res = attention_rows(K, V, Q, P, float(scale), rows, want_prob_sum)
-    return res + (K, V)
+    present = kept_mask(store, plan, layer, Kp.shape[1])
+    if present is None:
+        res = attention_rows(K, V, Q, P, float(scale), rows, want_prob_sum)
+        return res + (K, V)
+    # Compressed packets: kv head h simply does not have the pruned keys, so its q heads attend over the
+    # surviving prefix keys (in order) followed by the query block - one plain attention per kv head.
+    Hkv = Kp.shape[1]
+    g = Hq // Hkv
+    if rows is None:
+        rows = [(h, i) for i in range(q_len) for h in range(Hq)]
+    out = np.empty((len(rows), d), dtype=np.float64)
+    lse = np.empty((len(rows),), dtype=np.float64)
+    ps = np.empty((len(rows),), dtype=np.float64)
+    for hk in range(Hkv):
+        sel = [n for n, (h, i) in enumerate(rows) if h // g == hk]
+        if not sel:
+            continue
+        idx = np.nonzero(present[:, hk])[0]
+        Kh = np.concatenate([Kp[idx, hk:hk + 1], Kn[:, hk:hk + 1]], axis=0)
+        Vh = np.concatenate([Vp[idx, hk:hk + 1], Vn[:, hk:hk + 1]], axis=0)
+        sub = [(rows[n][0] - hk * g, rows[n][1]) for n in sel]
+        o, l, s_ = attention_rows(Kh, Vh, Q[:, hk * g:(hk + 1) * g], len(idx), float(scale), sub, True)
+        out[sel], lse[sel], ps[sel] = o, l, s_
+    if want_prob_sum:
+        return out, lse, ps, K, V
+    return out, lse, K, V
+
+
+def kept_mask(store: Store, plan: Plan, layer: int, n_kv_heads: int):
+    """present[t][h]: does kv head h of this layer still hold the key at composed position t?  None when
+    the request has no compressed packet (everything is present)."""
+    if not any(kind == "packet" and ident in store.kept for kind, ident in plan.refs):
+        return None
+    present = np.ones((plan.prefix_len, n_kv_heads), dtype=bool)
+    for (row0, n, t0, _), (kind, ident) in zip(plan.segments, plan.refs):
+        if kind == "packet" and ident in store.kept:
+            present[t0:t0 + n] = False
+            for h in range(n_kv_heads):
+                present[t0 + np.asarray(store.kept[ident][layer][h], dtype=np.int64), h] = True
+    return present

@@ -38,6 +38,7 @@ class kvp_config(ctypes.Structure):
         ("workspace_bytes", ctypes.c_uint64), ("max_packets", ctypes.c_int32), ("max_adapters", ctypes.c_int32),
         ("max_batch", ctypes.c_int32), ("max_slots", ctypes.c_int32), ("max_prefix_tokens", ctypes.c_int32),
         ("max_query_tokens", ctypes.c_int32), ("max_ws_rows", ctypes.c_int32), ("max_assemblies", ctypes.c_int32),
+        ("max_compressed", ctypes.c_int32),
     ]
 
 
@@ -63,6 +64,7 @@ def lib() -> ctypes.CDLL:
         "kvp_create": (i32, [pcfg, ctypes.POINTER(vp)]),
         "kvp_destroy": (i32, [vp]),
         "kvp_register_packet": (i32, [vp, vp, vp, i32, i32, vp, pi32]),
+        "kvp_register_packet_compressed": (i32, [vp, vp, vp, i32, i32, pi32, vp, pi32]),
         "kvp_register_adapter": (i32, [vp, vp, vp, i32, i32, vp, vp, i32, i32, vp, pi32]),
         "kvp_assemble": (i32, [vp, i32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
         "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
@@ -86,7 +88,7 @@ def lib() -> ctypes.CDLL:
 
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
-            "kvp_register_packet", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
+            "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
             "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
@@ -112,7 +114,8 @@ class Context:
                  rope_theta: float = 10000.0, rope_pairing: int = 0, softmax_scale: float = 0.0,
                  inv_freq: Optional[Sequence[float]] = None, pool_tokens: int = 0, max_packets: int = 64,
                  max_adapters: int = 4, max_batch: int = 1, max_slots: int = 64, max_prefix_tokens: int = 4096,
-                 max_query_tokens: int = 128, max_ws_rows: int = 0, max_assemblies: int = 1, device: int = 0):
+                 max_query_tokens: int = 128, max_ws_rows: int = 0, max_assemblies: int = 1, device: int = 0,
+                 max_compressed: int = 0):
         self._L = lib()
         self._h = ctypes.c_void_p()
         cfg = kvp_config()
@@ -132,6 +135,7 @@ class Context:
         if max_ws_rows <= 0:
             max_ws_rows = max_batch * max_query_tokens + 64 * max_slots
         cfg.max_ws_rows, cfg.max_assemblies = max_ws_rows, max_assemblies
+        cfg.max_compressed = max_compressed
         self.dtype, self.device = dtype, device
         self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
         self.token_bytes = int(self._L.kvp_token_bytes(ctypes.byref(cfg)))
@@ -183,6 +187,13 @@ class Context:
         out = ctypes.c_int32(-1)
         self._check(self._L.kvp_register_packet(self._h, _ptr(k), _ptr(v), n_tokens, cache_pos0,
                                                 self._stream(stream), ctypes.byref(out)))
+        return out.value
+
+    def register_packet_compressed(self, k, v, n_tokens: int, cache_pos0: int, kept: Sequence[int], stream=None) -> int:
+        """kept: n_layers * n_kv_heads row counts; k, v: the kept rows of every (layer, kv head), runs back to back."""
+        out = ctypes.c_int32(-1)
+        self._check(self._L.kvp_register_packet_compressed(self._h, _ptr(k), _ptr(v), n_tokens, cache_pos0,
+                                                           _i32_array(list(kept)), self._stream(stream), ctypes.byref(out)))
         return out.value
 
     def register_adapter(self, hk, hv, n_header: int, header_pos0: int, tk, tv, n_trailer: int,

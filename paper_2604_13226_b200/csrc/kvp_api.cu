@@ -58,23 +58,28 @@ bool valid_cfg(const kvp_config *c)
     if (c->max_prefix_tokens <= 0 || c->max_query_tokens <= 0 || c->max_ws_rows <= 0 || c->max_assemblies <= 0)
         return false;
     if (!c->inv_freq && !(c->rope_theta > 0.0)) return false;
+    if (c->max_compressed < 0) return false;
     return true;
 }
 
 kvp_plan_layout plan_layout(const kvp_config *c)
 {
     kvp_plan_layout p;
+    // with compressed packets every layer has its own item records and tile list
+    const int64_t lists = c->max_compressed > 0 ? c->n_layers : 1;
     p.max_segs = 3 * c->max_slots;
     p.max_rope = p.max_segs + 1;
-    p.max_tiles = c->max_batch * (c->max_prefix_tokens / KVP_TILE_KEYS + 2) + c->max_slots +
-                  c->max_ws_rows / KVP_TILE_KEYS + 8;
+    p.max_items = (int32_t)(c->max_batch * lists);
+    p.max_tiles = (int32_t)((c->max_batch * ((int64_t)c->max_prefix_tokens / KVP_TILE_KEYS + 2) + c->max_slots +
+                             c->max_ws_rows / KVP_TILE_KEYS + 8) * lists);
     p.max_chunks = c->max_ws_rows / KVP_CHUNK_ROWS + p.max_segs + 8;
     uint64_t o = 0;
-    p.items = o;  o = round_up(o + sizeof(kvp_item) * c->max_batch, 256);
-    p.tiles = o;  o = round_up(o + sizeof(kvp_tile) * p.max_tiles, 256);
+    p.items = o;  o = round_up(o + sizeof(kvp_item) * p.max_items, 256);
+    p.tiles = o;  o = round_up(o + sizeof(kvp_tile) * (uint64_t)p.max_tiles, 256);
     p.chunks = o; o = round_up(o + sizeof(kvp_chunk) * p.max_chunks, 256);
     p.segs = o;   o = round_up(o + sizeof(kvp_seg) * p.max_segs, 256);
     p.rope = o;   o = round_up(o + sizeof(float2) * (uint64_t)p.max_rope * (c->head_dim / 2), 256);
+    p.kept = o;   o = round_up(o + 4ull * c->max_compressed * c->n_layers * c->n_kv_heads, 256);
     p.total = o;
     return p;
 }
@@ -90,7 +95,7 @@ ws_layout workspace_layout(const kvp_config *c)
     w.rows_bytes = round_up((uint64_t)c->n_layers * c->n_kv_heads * c->max_ws_rows * c->head_dim * e, kAlign);
     w.slot_plan = 0;
     w.slot_sched = round_up(p.total, kAlign);
-    w.slot_k = round_up(w.slot_sched + schedule_layout(c).total, kAlign);
+    w.slot_k = round_up(w.slot_sched + schedule_layout(c).total * (c->max_compressed > 0 ? c->n_layers : 1), kAlign);
     w.slot_v = w.slot_k + w.rows_bytes;
     w.slot_stride = w.slot_v + w.rows_bytes;
     w.slots = o;    o += w.slot_stride * c->max_assemblies;
@@ -164,6 +169,9 @@ kvp_plan_dev plan_dev(const kvp_ctx *ctx, int slot)
     p.chunks = reinterpret_cast<const kvp_chunk *>(base + ctx->pl.chunks);
     p.segs = reinterpret_cast<const kvp_seg *>(base + ctx->pl.segs);
     p.rope = reinterpret_cast<const float2 *>(base + ctx->pl.rope);
+    p.kept = reinterpret_cast<const int32_t *>(base + ctx->pl.kept);
+    p.item_stride = ctx->slots[slot].item_stride;
+    p.n_planes = ctx->shape.n_layers * ctx->shape.n_kv_heads;
     return p;
 }
 
@@ -189,7 +197,7 @@ struct schedule_t {
     int32_t n_ctas = 0, n_slots = 0, max_pieces = 1;
 };
 
-int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, int q_pos0, schedule_t &out)
+int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int q_len, int q_pos0, schedule_t &out)
 {
     const kvp_shape &sh = ctx->shape;
     struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces; };
@@ -197,7 +205,8 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, int 
     const int n_rows = sh.group * q_len;
     int64_t total = 0;
     for (int b = 0; b < as.batch; ++b) {
-        const int n_prefix = as.items[b].tile_end - as.items[b].tile_begin;
+        const kvp_item &item = as.items[(as.item_stride ? layer * as.item_stride : 0) + b];
+        const int n_prefix = item.tile_end - item.tile_begin;
         for (int hk = 0; hk < sh.n_kv_heads; ++hk)
             for (int row_base = 0; row_base < n_rows; row_base += 2 * KVP_TILE_ROWS) {
                 unit_t u;
@@ -312,10 +321,10 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int q_len, int 
     return KVP_OK;
 }
 
-int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len, int q_pos0, cudaStream_t st)
+int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer, int q_len, int q_pos0, cudaStream_t st)
 {
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, as, q_len, q_pos0, sc);
+    const int32_t rc = plan_schedule(ctx, as, layer, q_len, q_pos0, sc);
     if (rc != KVP_OK) return rc;
     const std::vector<int32_t> &cta_begin = sc.cta_begin;
     const std::vector<kvp_work> &works = sc.works;
@@ -327,7 +336,8 @@ int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len,
     memcpy(h, cta_begin.data(), 4 * cta_begin.size());
     memcpy(h + ctx->sched_off_works, works.data(), sizeof(kvp_work) * works.size());
     memcpy(h + ctx->sched_off_merges, merges.data(), sizeof(kvp_merge_item) * merges.size());
-    char *d = ctx->slot_sched_dev[slot];
+    const int li = as.item_stride ? layer : 0;                   // which of the assembly's work lists
+    char *d = ctx->slot_sched_dev[slot] + ctx->sched_bytes * li;
     KVP_CUDA(ctx, cudaMemcpyAsync(d, h, 4 * cta_begin.size(), cudaMemcpyHostToDevice, st));
     KVP_CUDA(ctx, cudaMemcpyAsync(d + ctx->sched_off_works, h + ctx->sched_off_works, sizeof(kvp_work) * works.size(),
                                   cudaMemcpyHostToDevice, st));
@@ -335,12 +345,13 @@ int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int q_len,
         KVP_CUDA(ctx, cudaMemcpyAsync(d + ctx->sched_off_merges, h + ctx->sched_off_merges,
                                       sizeof(kvp_merge_item) * merges.size(), cudaMemcpyHostToDevice, st));
     KVP_CUDA(ctx, cudaEventRecord(ctx->sched_event[slot], st));
-    as.sched_q_len = q_len;
-    as.sched_q_pos0 = q_pos0;
-    as.sched_ctas = n_ctas;
-    as.sched_works = (int32_t)works.size();
-    as.sched_merges = (int32_t)merges.size();
-    as.sched_slots = max_pieces;
+    kvp_assembly_host::sched_state &ss = as.sched[li];
+    ss.q_len = q_len;
+    ss.q_pos0 = q_pos0;
+    ss.ctas = n_ctas;
+    ss.works = (int32_t)works.size();
+    ss.merges = (int32_t)merges.size();
+    ss.slots = max_pieces;
     return KVP_OK;
 }
 
@@ -521,8 +532,44 @@ int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t 
     if (ctx->pool_rows_used + n_tokens > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
     const int32_t rc = store_segment(ctx, k, v, n_tokens, (cudaStream_t)stream);
     if (rc != KVP_OK) return rc;
-    ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0});
+    ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0, {}});
     ctx->pool_rows_used += n_tokens;
+    *packet_id = (int32_t)ctx->packets.size() - 1;
+    return KVP_OK;
+}
+
+int32_t kvp_register_packet_compressed(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens,
+                                       int32_t cache_pos0, const int32_t *kept, void *stream, int32_t *packet_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!packet_id || !kept || n_tokens <= 0) return fail(ctx, KVP_ERR_INVALID, "register_packet_compressed: bad arguments");
+    if (ctx->cfg.max_compressed <= 0) return fail(ctx, KVP_ERR_STATE, "register_packet_compressed: max_compressed is 0");
+    if (!ctx->host_only && (!k || !v)) return fail(ctx, KVP_ERR_INVALID, "register_packet_compressed: null K/V");
+    if ((int)ctx->packets.size() >= ctx->cfg.max_packets) return fail(ctx, KVP_ERR_CAPACITY, "max_packets reached");
+    const kvp_shape &sh = ctx->shape;
+    const int planes = sh.n_layers * sh.n_kv_heads;
+    int32_t n_max = 0;
+    for (int i = 0; i < planes; ++i) {
+        if (kept[i] < 1 || kept[i] > n_tokens) return fail(ctx, KVP_ERR_INVALID, "register_packet_compressed: kept[%d] = %d", i, kept[i]);
+        n_max = std::max(n_max, kept[i]);
+    }
+    if (ctx->pool_rows_used + n_max > sh.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
+    if (!ctx->host_only) {
+        // plane (l, h) receives its run of kept rows; the runs lie back to back in the caller's buffers
+        cudaStream_t st = (cudaStream_t)stream;
+        KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+        const size_t row_bytes = (size_t)sh.head_dim * sh.elem_bytes;
+        size_t src_off = 0;
+        for (int i = 0; i < planes; ++i) {
+            const size_t dst_off = ((size_t)i * sh.pool_rows + ctx->pool_rows_used) * row_bytes;
+            const size_t n = (size_t)kept[i] * row_bytes;
+            KVP_CUDA(ctx, cudaMemcpyAsync(ctx->pool_k + dst_off, (const char *)k + src_off, n, cudaMemcpyDeviceToDevice, st));
+            KVP_CUDA(ctx, cudaMemcpyAsync(ctx->pool_v + dst_off, (const char *)v + src_off, n, cudaMemcpyDeviceToDevice, st));
+            src_off += n;
+        }
+    }
+    ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0, std::vector<int32_t>(kept, kept + planes)});
+    ctx->pool_rows_used += n_max;
     *packet_id = (int32_t)ctx->packets.size() - 1;
     return KVP_OK;
 }
@@ -539,11 +586,11 @@ int32_t kvp_register_adapter(kvp_ctx *ctx, const void *hk, const void *hv, int32
     if (ctx->pool_rows_used + n_header + n_trailer > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
     int32_t rc = store_segment(ctx, hk, hv, n_header, (cudaStream_t)stream);
     if (rc != KVP_OK) return rc;
-    ctx->adapter_h.push_back({(int32_t)ctx->pool_rows_used, n_header, header_pos0});
+    ctx->adapter_h.push_back({(int32_t)ctx->pool_rows_used, n_header, header_pos0, {}});
     ctx->pool_rows_used += n_header;
     rc = store_segment(ctx, tk, tv, n_trailer, (cudaStream_t)stream);
     if (rc != KVP_OK) { ctx->adapter_h.pop_back(); ctx->pool_rows_used -= n_header; return rc; }
-    ctx->adapter_t.push_back({(int32_t)ctx->pool_rows_used, n_trailer, trailer_pos0});
+    ctx->adapter_t.push_back({(int32_t)ctx->pool_rows_used, n_trailer, trailer_pos0, {}});
     ctx->pool_rows_used += n_trailer;
     *adapter_id = (int32_t)ctx->adapter_h.size() - 1;
     return KVP_OK;
@@ -586,10 +633,17 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
         for (int32_t o = 0; o < n; o += KVP_CHUNK_ROWS)
             chunks.push_back({src + o, dst + o, std::min<int32_t>(KVP_CHUNK_ROWS, n - o), rope});
     };
-    auto add_tiles = [&](int16_t src, int32_t row0, int32_t n, int32_t rope, int32_t pos0) {
+    // kept_row < 0: every plane holds all n rows; else the run belongs to a compressed packet whose
+    // per-plane counts are row kept_row of the assembly's table, and n is the largest of this layer's
+    auto add_tiles = [&](int16_t src, int32_t row0, int32_t n, int32_t rope, int32_t kept_row) {
         for (int32_t o = 0; o < n; o += KVP_TILE_KEYS)
-            as.tiles.push_back({row0 + o, (int16_t)std::min<int32_t>(KVP_TILE_KEYS, n - o), src, rope, pos0 + o});
+            as.tiles.push_back({row0 + o, (int16_t)std::min<int32_t>(KVP_TILE_KEYS, n - o), src, rope,
+                                kept_row < 0 ? -1 : (kept_row << 16) | (o / KVP_TILE_KEYS)});
     };
+    std::map<int32_t, int32_t> kept_row_of;    // compressed packet id -> row of the kept table
+    std::vector<int32_t> kept_packets;
+    struct item_build { kvp_item it; int32_t stage0, staged; };
+    std::vector<item_build> builds;
 
     for (int b = 0; b < batch; ++b) {
         kvp_item it;
@@ -620,6 +674,15 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
                 e.rope = f->second;
                 e.pad[0] = -1;                   // workspace row of a staged copy, if any
                 e.pad[1] = k;                    // 0 header, 1 document, 2 trailer
+                e.pad[2] = -1;                   // row of the kept table (compressed document)
+                if (k == 1 && !sg->kept.empty()) {
+                    auto kr = kept_row_of.find(packet_ids[s]);
+                    if (kr == kept_row_of.end()) {
+                        kr = kept_row_of.emplace(packet_ids[s], (int32_t)kept_packets.size()).first;
+                        kept_packets.push_back(packet_ids[s]);
+                    }
+                    e.pad[2] = kr->second;
+                }
                 if (!mat && k != 1) staged += sg->n;
                 as.segs.push_back(e);
                 t += sg->n;
@@ -629,16 +692,19 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
         it.seg_end = (int32_t)as.segs.size();
         it.prefix_len = (int32_t)t;
         prefix_len[b] = (int32_t)t;
-        it.tile_begin = (int32_t)as.tiles.size();
         if (mat) {
+            if (!kept_packets.empty()) return fail(ctx, KVP_ERR_UNSUPPORTED, "assemble: compressed packets cannot be materialised");
+            it.tile_begin = (int32_t)as.tiles.size();
             it.cache_row0 = (int32_t)ws_cursor;
             for (int s = it.seg_begin; s < it.seg_end; ++s) {
                 kvp_seg &e = as.segs[s];
                 add_chunks(e.src_row0, it.cache_row0 + e.dst_pos0, e.len, e.rope);
             }
-            add_tiles(1, it.cache_row0, it.prefix_len, 0, 0);
+            add_tiles(1, it.cache_row0, it.prefix_len, 0, -1);
             it.tail_row0 = it.cache_row0 + it.prefix_len;
+            it.tile_end = (int32_t)as.tiles.size();
             ws_cursor += (int64_t)it.prefix_len + cfg.max_query_tokens;
+            builds.push_back({it, 0, 0});
         } else {
             it.cache_row0 = -1;
             const int32_t stage0 = (int32_t)ws_cursor;
@@ -650,19 +716,42 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
                 add_chunks(e.src_row0, e.pad[0], e.len, e.rope);
                 so += e.len;
             }
-            add_tiles(1, stage0, so, 0, -1);
-            for (int s = it.seg_begin; s < it.seg_end; ++s) {      // documents: read in place
-                const kvp_seg &e = as.segs[s];
-                if (e.pad[1] == 1) add_tiles(0, e.src_row0, e.len, e.rope, e.dst_pos0);
-            }
             it.tail_row0 = stage0 + so;
             ws_cursor += (int64_t)so + cfg.max_query_tokens;
+            builds.push_back({it, stage0, so});
         }
-        it.tile_end = (int32_t)as.tiles.size();
         if (ws_cursor > cfg.max_ws_rows) return fail(ctx, KVP_ERR_CAPACITY, "assemble: needs more than max_ws_rows workspace rows");
-        as.items.push_back(it);
     }
+    if ((int)kept_packets.size() > cfg.max_compressed)
+        return fail(ctx, KVP_ERR_CAPACITY, "assemble: %zu compressed packets > max_compressed", kept_packets.size());
+    // tile lists: one for all layers, or - when a compressed packet keeps a different number of rows per
+    // layer - one per layer (documents are read in place; the staged adapter rows come first)
+    const int n_lists = kept_packets.empty() ? 1 : cfg.n_layers;
+    as.item_stride = kept_packets.empty() ? 0 : batch;
+    for (int l = 0; l < n_lists; ++l)
+        for (int b = 0; b < batch; ++b) {
+            kvp_item it = builds[b].it;
+            if (!mat) {
+                it.tile_begin = (int32_t)as.tiles.size();
+                add_tiles(1, builds[b].stage0, builds[b].staged, 0, -1);
+                for (int s = it.seg_begin; s < it.seg_end; ++s) {
+                    const kvp_seg &e = as.segs[s];
+                    if (e.pad[1] != 1) continue;
+                    if (e.pad[2] < 0) {
+                        add_tiles(0, e.src_row0, e.len, e.rope, -1);
+                    } else {
+                        const std::vector<int32_t> &kept = ctx->packets[kept_packets[e.pad[2]]].kept;
+                        int32_t n_l = 0;
+                        for (int h = 0; h < cfg.n_kv_heads; ++h) n_l = std::max(n_l, kept[l * cfg.n_kv_heads + h]);
+                        add_tiles(0, e.src_row0, n_l, e.rope, e.pad[2]);
+                    }
+                }
+                it.tile_end = (int32_t)as.tiles.size();
+            }
+            as.items.push_back(it);
+        }
     if ((int)as.tiles.size() > ctx->pl.max_tiles || (int)chunks.size() > ctx->pl.max_chunks ||
+        (int)as.items.size() > ctx->pl.max_items ||
         (int)rope_delta.size() > ctx->pl.max_rope || (int)as.segs.size() > ctx->pl.max_segs)
         return fail(ctx, KVP_ERR_CAPACITY, "assemble: plan tables overflow");
     as.n_chunks = (int32_t)chunks.size();
@@ -688,14 +777,26 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
             }
         const uint64_t used = ctx->pl.rope + sizeof(float2) * rope_delta.size() * half;
         KVP_CUDA(ctx, cudaMemcpyAsync(ctx->slot_plan_dev[slot], h, used, cudaMemcpyHostToDevice, st));
+        if (!kept_packets.empty()) {
+            const size_t planes = (size_t)cfg.n_layers * cfg.n_kv_heads;
+            int32_t *kt = reinterpret_cast<int32_t *>(h + ctx->pl.kept);
+            for (size_t r = 0; r < kept_packets.size(); ++r)
+                memcpy(kt + r * planes, ctx->packets[kept_packets[r]].kept.data(), 4 * planes);
+            KVP_CUDA(ctx, cudaMemcpyAsync(ctx->slot_plan_dev[slot] + ctx->pl.kept, kt, 4 * planes * kept_packets.size(),
+                                          cudaMemcpyHostToDevice, st));
+        }
         KVP_CUDA(ctx, cudaEventRecord(ctx->slot_event[slot], st));
+    }
+    const int32_t n_chunks = as.n_chunks;
+    ctx->slots[slot] = std::move(as);
+    *assembly_id = id;
+    if (!ctx->host_only) {
+        cudaStream_t st = (cudaStream_t)stream;
         KVP_CUDA(ctx, time_edge(ctx, 1, 0, st));
-        KVP_CUDA(ctx, kvp_launch_gather(ctx->shape, plan_dev(ctx, slot), as.n_chunks, ctx->pool_k, ctx->pool_v,
+        KVP_CUDA(ctx, kvp_launch_gather(ctx->shape, plan_dev(ctx, slot), n_chunks, ctx->pool_k, ctx->pool_v,
                                         ctx->slot_k[slot], ctx->slot_v[slot], st));
         KVP_CUDA(ctx, time_edge(ctx, 1, 1, st));
     }
-    ctx->slots[slot] = std::move(as);
-    *assembly_id = id;
     return KVP_OK;
 }
 
@@ -716,7 +817,7 @@ int32_t kvp_export_plan(kvp_ctx *ctx, int32_t assembly_id, int32_t b, int32_t *s
             row[0] = e.src_row0; row[1] = e.len; row[2] = e.dst_pos0; row[3] = e.delta;
         }
         for (int o = 0; o < e.len; ++o) {
-            if (src_row) src_row[e.dst_pos0 + o] = e.src_row0 + o;
+            if (src_row) src_row[e.dst_pos0 + o] = e.pad[2] >= 0 ? -1 : e.src_row0 + o;   // compressed: no row per position
             if (delta) delta[e.dst_pos0 + o] = e.delta;
         }
     }
@@ -731,6 +832,7 @@ int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32
     const int slot = find_slot(ctx, assembly_id);
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_cache: unknown assembly %d", assembly_id);
     const kvp_assembly_host &as = ctx->slots[slot];
+    if (as.item_stride) return fail(ctx, KVP_ERR_UNSUPPORTED, "export_cache: the assembly uses compressed packets");
     if (b < 0 || b >= as.batch || layer < 0 || layer >= ctx->cfg.n_layers || !k_out || !v_out || n_query_rows < 0 ||
         n_query_rows > ctx->cfg.max_query_tokens)
         return fail(ctx, KVP_ERR_INVALID, "export_cache: bad arguments");
@@ -782,17 +884,20 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         ++launches;
         ctx->last_kind = 0;
     } else if (ctx->kernel_variant == 0) {
-        if (as.sched_q_len != q_len || as.sched_q_pos0 != q_pos0 || as.sched_ctas == 0) {
-            const int32_t rc = build_schedule(ctx, as, slot, q_len, q_pos0, st);
+        const int li = as.item_stride ? layer : 0;
+        if (as.sched.empty()) as.sched.resize(as.item_stride ? ctx->cfg.n_layers : 1);
+        if (as.sched[li].q_len != q_len || as.sched[li].q_pos0 != q_pos0 || as.sched[li].ctas == 0) {
+            const int32_t rc = build_schedule(ctx, as, slot, layer, q_len, q_pos0, st);
             if (rc != KVP_OK) return rc;
         }
-        const char *sd = ctx->slot_sched_dev[slot];
+        const kvp_assembly_host::sched_state &ss = as.sched[li];
+        const char *sd = ctx->slot_sched_dev[slot] + ctx->sched_bytes * li;
         kvp_attn2_args a;
         a.plan = plan;
         a.q_len = q_len;
         a.q_pos0 = q_pos0;
         a.layer = layer;
-        a.n_ctas = as.sched_ctas;
+        a.n_ctas = ss.ctas;
         a.cta_begin = reinterpret_cast<const int32_t *>(sd);
         a.works = reinterpret_cast<const kvp_work *>(sd + ctx->sched_off_works);
         a.q = q_used;
@@ -805,17 +910,17 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot], ctx->tm_ws_v[slot], st));
         KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
-        if (as.sched_merges > 0) {
-            KVP_CUDA(ctx, kvp_launch_merge_list(sh, q_len, as.sched_merges,
+        if (ss.merges > 0) {
+            KVP_CUDA(ctx, kvp_launch_merge_list(sh, q_len, ss.merges,
                                                 reinterpret_cast<const kvp_merge_item *>(sd + ctx->sched_off_merges),
                                                 ctx->partial_o, ctx->partial_ml, out, lse, st));
             ++launches;
         }
-        ctas = as.sched_ctas;
-        splits = as.sched_slots;
+        ctas = ss.ctas;
+        splits = ss.slots;
         ctx->last_kind = 1;
     } else {
-        if (q_pos0 > 0) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: the single-tile kernel variant has no KVP_CONTINUE");
+        if (q_pos0 > 0 || as.item_stride) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: the single-tile kernel variant has no KVP_CONTINUE and no compressed packets");
         const int n_mtiles = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
         const int units = as.batch * sh.n_kv_heads * n_mtiles;
         int min_tiles = INT32_MAX;
@@ -891,7 +996,7 @@ int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, in
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_schedule: unknown assembly %d", assembly_id);
     if (q_len <= 0 || q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_INVALID, "export_schedule: bad q_len");
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], q_len, 0, sc);
+    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], 0, q_len, 0, sc);
     if (rc != KVP_OK) return rc;
     counts[0] = sc.n_ctas;
     counts[1] = (int32_t)sc.works.size();
@@ -924,7 +1029,7 @@ int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
     if (!ctx) return KVP_ERR_INVALID;
     if (key == KVP_TUNE_SPLIT_TARGET_CTAS || key == KVP_TUNE_FORCE_SPLITS) {
         (key == KVP_TUNE_SPLIT_TARGET_CTAS ? ctx->split_target_ctas : ctx->force_splits) = value;
-        for (kvp_assembly_host &as : ctx->slots) as.sched_q_len = 0;      // work lists are rebuilt on next use
+        for (kvp_assembly_host &as : ctx->slots) as.sched.clear();       // work lists are rebuilt on next use
     }
     else if (key == KVP_TUNE_KERNEL_VARIANT) {
         if (value != 0 && value != 1) return fail(ctx, KVP_ERR_INVALID, "tune: kernel variant %d", value);

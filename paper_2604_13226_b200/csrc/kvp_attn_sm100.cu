@@ -275,7 +275,7 @@ __device__ __forceinline__ Work load_work(const Params &p, int wi)
     Work w;
     w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w;
     w.lo = c.x; w.n = c.y; w.slot0 = c.z; w.slot1 = c.w;
-    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + w.b);
+    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + p.layer * p.plan.item_stride + w.b);
     const int4 ia = __ldg(i4), ib = __ldg(i4 + 1);          // prefix_len, tile_begin, tile_end, seg_begin | seg_end, tail_row0, ..
     w.tile_begin = ia.y;
     w.tail_row0 = ib.y;
@@ -309,6 +309,10 @@ __device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
         t.src = g.y >> 16;
         t.rope = g.z;
         t.qoff = -1;
+        if (g.w >= 0) {        // compressed packet: this (layer, kv head) keeps fewer rows, possibly none of this tile
+            const int kept = __ldg(p.plan.kept + (g.w >> 16) * p.plan.n_planes + w.plane);
+            t.n_keys = max(0, min(t.n_keys, kept - (g.w & 0xFFFF) * KVP_TILE_KEYS));
+        }
     }
     return t;
 }
@@ -772,7 +776,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
         ok = __all_sync(0xffffffffu, ok);                         // the lanes stay together
         if (!ok) return;
         tc_fence_after();
-        const uint32_t n16 = (uint32_t)(tl.n_keys + 15) & ~15u;
+        const uint32_t n16 = max(16u, (uint32_t)(tl.n_keys + 15) & ~15u);      // a tile may be empty for this head
         const uint32_t idesc = instr_desc(n16, 0);
         const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
         const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
@@ -823,7 +827,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                     for (int kk = 0; kk < 8; ++kk)               // 16 keys per step: P advances 8 columns, V 2048 bytes
                         mma_ts_c<1>(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv);
                 } else {
-                    const int ksteps = (ms.prev_keys + 15) >> 4;
+                    const int ksteps = max(1, (ms.prev_keys + 15) >> 4);   // an empty tile still initialises O (P = 0)
                     for (int kk = 0; kk < ksteps; ++kk)
                         mma_ts(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv, (k > 1 || kk > 0));
                 }

@@ -22,7 +22,8 @@ struct kvp_tile {              // one run of <= 128 consecutive key rows sharing
     int16_t n_keys;            // 1..128
     int16_t src;               // 0 pool, 1 workspace
     int32_t rope;              // rope-table index of the offset still to be applied to these keys (0 = none)
-    int32_t pos0;              // composed position of the first key (diagnostics)
+    int32_t clip;              // -1, or (row of the kept-count table << 16) | tile number inside the packet:
+                               // plane (layer, kv head) then holds only kept - 128 * tile number of these keys
 };
 
 struct kvp_chunk {             // gather work item: <= 32 rows copied pool -> workspace, keys rotated
@@ -75,8 +76,8 @@ struct kvp_merge_item {        // 128 packed rows whose result is spread over n_
 
 // Offsets (bytes) of the arrays inside one plan blob; identical on host and device.
 struct kvp_plan_layout {
-    uint64_t items, tiles, chunks, segs, rope, total;
-    int32_t max_tiles, max_chunks, max_segs, max_rope;
+    uint64_t items, tiles, chunks, segs, rope, kept, total;
+    int32_t max_items, max_tiles, max_chunks, max_segs, max_rope;
 };
 
 // Pointers into a device-resident plan, passed to kernels by value.
@@ -86,6 +87,9 @@ struct kvp_plan_dev {
     const kvp_chunk *chunks;
     const kvp_seg *segs;
     const float2 *rope;        // [n_rope][head_dim/2] (cos, sin) of delta * theta_i
+    const int32_t *kept;       // [compressed packets of the assembly][n_layers * n_kv_heads] kept rows per plane
+    int32_t item_stride;       // 0: one item / tile list for all layers; batch: items[layer * batch + b]
+    int32_t n_planes;
 };
 
 struct kvp_shape {
@@ -97,7 +101,10 @@ struct kvp_shape {
 
 // ---- host-side context -----------------------------------------------------------------------
 
-struct kvp_segment_host { int32_t row0, n, pos0; };
+struct kvp_segment_host {
+    int32_t row0, n, pos0;             // first pool row, positions covered, position it was cached at
+    std::vector<int32_t> kept;         // compressed packets: rows kept per plane (layer, kv head); else empty
+};
 
 struct kvp_assembly_host {
     int32_t id = -1;
@@ -107,11 +114,13 @@ struct kvp_assembly_host {
     std::vector<kvp_seg> segs;
     std::vector<kvp_tile> tiles;
     int32_t n_chunks = 0, n_rope = 0;
+    int32_t item_stride = 0;               // batch when the assembly has per-layer tile lists (compressed packets)
     int32_t last_q_len = 0;
     std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
-    // work list of the two-stream kernel, built for sched_q_len query tokens at offset sched_q_pos0 (0 = none yet)
-    int32_t sched_q_pos0 = 0;
-    int32_t sched_q_len = 0, sched_ctas = 0, sched_works = 0, sched_merges = 0, sched_slots = 0;
+    // work lists of the two-stream kernel (one, or one per layer when the tile lists differ per layer), each
+    // built for q_len query tokens at offset q_pos0 (q_len 0 = none yet)
+    struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; };
+    std::vector<sched_state> sched;
 };
 
 struct kvp_ctx {

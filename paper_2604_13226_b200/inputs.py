@@ -88,6 +88,7 @@ class Packet:
     k: np.ndarray                  # [n_layers][n_tokens][n_kv_heads][head_dim], stored dtype
     v: np.ndarray
     cache_pos0: int = 0
+    kept: Optional[list] = None    # compressed packet: kept[layer][kv_head] = sorted token indices that survive pruning
 
     @property
     def n_tokens(self) -> int:
@@ -170,6 +171,8 @@ def make_workload(shape: ModelShape,
                   adapter_pos0: Optional[Sequence[Tuple[int, int]]] = None,
                   outlier_channels: int = 0,
                   outlier_scale: float = 8.0,
+                  keep_rate: Optional[Sequence[Optional[float]]] = None,
+                  keep_per_head: bool = True,
                   name: str = "") -> Workload:
     """Draw a workload with ``numpy.random.default_rng(seed)``.
 
@@ -179,6 +182,10 @@ def make_workload(shape: ModelShape,
     stated std, then narrowed to the stored dtype.  ``outlier_channels`` > 0 multiplies that
     many seeded channels per (layer, kv head) of every packet's K and V by ``outlier_scale``
     before narrowing (same channels for all packets).
+    ``keep_rate[p]`` (None = not compressed) marks packet p as pruned: a stand-in for an unstructured
+    KV compressor, every (layer, kv head) keeps a seeded random subset of the tokens, about that
+    fraction of them - a different count per head with ``keep_per_head``, else one count per layer.
+    These draws come from their own generator, after everything else.
     """
     rng = np.random.default_rng(seed)
     L, Hq, Hkv, d = shape.n_layers, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
@@ -220,6 +227,21 @@ def make_workload(shape: ModelShape,
     wl = Workload(shape, packets, adapters, [list(map(tuple, it)) for it in items], q, k_new, v_new,
                   rebase=rebase, name=name, seed=seed)
     wl.notes["chan_scale"] = chan_scale        # [L][1][Hkv][d] multipliers applied to packet K/V, or None
+    if keep_rate is not None:
+        krng = np.random.default_rng(seed + 104729)
+        for i, rate in enumerate(keep_rate):
+            if rate is None:
+                continue
+            n = packets[i].n_tokens
+            kept = []
+            for l in range(L):
+                n_layer = max(1, min(n, int(round(n * rate * krng.uniform(0.7, 1.3)))))
+                row = []
+                for h in range(Hkv):
+                    n_h = max(1, min(n, int(round(n_layer * krng.uniform(0.6, 1.0))))) if keep_per_head else n_layer
+                    row.append(np.sort(krng.choice(n, size=n_h, replace=False)).astype(np.int64))
+                kept.append(row)
+            packets[i].kept = kept
     return wl
 
 

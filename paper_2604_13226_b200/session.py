@@ -62,7 +62,8 @@ class Session:
                                rope_pairing=s.rope_pairing, pool_tokens=sum(lens) + ad_tokens + 8,
                                max_packets=len(lens), max_adapters=max(1, n_adapters), max_batch=B,
                                max_slots=max(1, n_slots), max_prefix_tokens=max(prefix + [1]), max_query_tokens=mq,
-                               max_ws_rows=ws_rows + 8, max_assemblies=max_assemblies, device=device)
+                               max_ws_rows=ws_rows + 8, max_assemblies=max_assemblies, device=device,
+                               max_compressed=0 if is_dev else sum(1 for p in wl.packets if p.kept is not None))
         # registration (offline in the paper; not part of any timed region)
         if is_dev:
             for pid in range(len(lens)):
@@ -73,6 +74,15 @@ class Session:
             self.ctx.register_adapter(hk, hv, wl.spec.n_header, 0, tk, tv, wl.spec.n_trailer, 0)
         else:
             for p in wl.packets:
+                if p.kept is not None:
+                    # the compressor's output: for every (layer, kv head) its surviving rows, runs back to back
+                    runs_k = [p.k[l][p.kept[l][h], h, :] for l in range(s.n_layers) for h in range(s.n_kv_heads)]
+                    runs_v = [p.v[l][p.kept[l][h], h, :] for l in range(s.n_layers) for h in range(s.n_kv_heads)]
+                    counts = [len(p.kept[l][h]) for l in range(s.n_layers) for h in range(s.n_kv_heads)]
+                    k = np_to_torch(np.concatenate(runs_k, axis=0), s.dtype, self.device)
+                    v = np_to_torch(np.concatenate(runs_v, axis=0), s.dtype, self.device)
+                    self.ctx.register_packet_compressed(k, v, p.n_tokens, p.cache_pos0, counts)
+                    continue
                 k = np_to_torch(p.k, s.dtype, self.device)
                 v = np_to_torch(p.v, s.dtype, self.device)
                 self.ctx.register_packet(k, v, p.n_tokens, p.cache_pos0)

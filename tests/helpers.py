@@ -16,7 +16,7 @@ def make_store(wl):
                             (lambda layer: (ad.hk[layer], ad.hv[layer], ad.tk[layer], ad.tv[layer])))
         return st
     for p in wl.packets:
-        st.register_packet(p.n_tokens, p.cache_pos0, (lambda layer, p=p: (p.k[layer], p.v[layer])))
+        st.register_packet(p.n_tokens, p.cache_pos0, (lambda layer, p=p: (p.k[layer], p.v[layer])), kept=p.kept)
     for a in wl.adapters:
         st.register_adapter(a.n_header, a.header_pos0, a.n_trailer, a.trailer_pos0,
                             (lambda layer, a=a: (a.hk[layer], a.hv[layer], a.tk[layer], a.tv[layer])))

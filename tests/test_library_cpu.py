@@ -199,3 +199,29 @@ def test_schedule_covers_every_tile_once(case):
     # balance: no CTA carries more than its share plus a few tiles (a piece's fixed cost counts as 8)
     cost = [sum(int(works[i][5]) * (1 if works[i][3] else 2) + 8 for i in range(cb[c], cb[c + 1])) for c in range(len(cb) - 1)]
     assert max(cost) <= sum(cost) / len(cost) + 16
+
+
+def test_compressed_registration_and_per_layer_lists_host_only():
+    shape = gen.ModelShape(3, 8, 2, 128, "bf16", 500000.0)
+    wl = gen.make_workload(shape, [300, 700], [[(0, 0), (1, 0)]], q_len=8, seed=2, keep_rate=[0.5, None])
+    ctx = kvp.Context(3, 8, 2, 128, "bf16", rope_theta=500000.0, max_packets=4, max_adapters=1, max_batch=1, max_slots=2,
+                      max_prefix_tokens=1100, max_query_tokens=8, max_ws_rows=200, device=-1, max_compressed=1)
+    counts = [len(wl.packets[0].kept[l][h]) for l in range(3) for h in range(2)]
+    pid = ctx.register_packet_compressed(None, None, 300, 0, counts)
+    ctx.register_packet(None, None, 700, 0)
+    ctx.register_adapter(None, None, 16, 0, None, None, 16, 0)
+    aid, plen = ctx.assemble(wl.items, kvp.REBASE)
+    assert pid == 0 and plen == [16 + 300 + 16 + 16 + 700 + 16]
+    src, dl, segs = ctx.export_plan(aid, 0)
+    assert np.all(src[16:316] == -1) and np.all(dl[16:316] == 16)       # one offset for the compressed packet
+    assert src[348] == max(counts)                                       # the next packet follows max(kept) pool rows
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.register_packet_compressed(None, None, 300, 0, [0] * 6)
+    assert e.value.code == 1
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.register_packet_compressed(None, None, 300, 0, [301] * 6)
+    assert e.value.code == 1
+    plain = kvp.Context(3, 8, 2, 128, "bf16", max_packets=2, device=-1)
+    with pytest.raises(kvp.KvpError) as e:
+        plain.register_packet_compressed(None, None, 300, 0, counts)
+    assert e.value.code == 4

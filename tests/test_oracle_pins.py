@@ -10,6 +10,7 @@ import pytest
 from oracle import bruteforce as bf
 from oracle import reference as orc
 from paper_2604_13226_b200 import inputs as gen
+from helpers import oracle_outputs
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -330,3 +331,81 @@ def test_widen_bf16_exact():
     assert list(orc.widen(bits, "bf16")) == [1.0, -1.0, 3.140625, 0.0, float(np.float32(3.3895314e38))]
     x = np.array([1.0, 1.00390625, 1.001953125, 1.005859375], dtype=np.float32)   # ties-to-even cases
     assert list(gen.f32_to_bf16_bits(x)) == [0x3F80, 0x3F80, 0x3F80, 0x3F81]
+
+
+# ------------------------------------------------------------------------------------------------
+# compressed packets (Section 4.3): a kv head attends over the keys its pruned cache still holds
+# ------------------------------------------------------------------------------------------------
+
+def _compressed_case(keep_rate, seed=11, q_len=6, dtype="f32"):
+    shape = gen.ModelShape(2, 4, 2, 64, dtype, 10000.0, 0)
+    return gen.make_workload(shape, [50, 33, 70], [[(0, 0), (1, 0), (2, -1)]], q_len=q_len, n_header=3, n_trailer=2,
+                             seed=seed, keep_rate=keep_rate, packet_pos0=[0, 4, 0])
+
+
+def test_compressed_keep_everything_equals_uncompressed():
+    wl = _compressed_case([None, None, None])
+    ref = oracle_outputs(wl, layer=1)[0]
+    for p in wl.packets:
+        p.kept = [[np.arange(p.n_tokens) for _ in range(2)] for _ in range(2)]
+    got = oracle_outputs(wl, layer=1)[0]
+    assert np.array_equal(got[0], ref[0]) and np.array_equal(got[1], ref[1])
+
+
+def test_compressed_equals_masked_dense_attention():
+    # independent route: dense scores over the whole composed sequence, pruned keys masked to -inf
+    wl = _compressed_case([0.5, None, 0.3])
+    s = wl.shape
+    for layer in range(s.n_layers):
+        out, lse, K, V, plan = oracle_outputs(wl, layer=layer)[0]
+        P = plan.prefix_len
+        present = np.ones((P + wl.q_len, s.n_kv_heads), dtype=bool)
+        t = 0
+        for pid, aid in wl.items[0]:
+            if aid >= 0:
+                t += wl.adapters[aid].n_header
+            p = wl.packets[pid]
+            if p.kept is not None:
+                present[t:t + p.n_tokens] = False
+                for h in range(s.n_kv_heads):
+                    present[t + p.kept[layer][h], h] = True
+            t += p.n_tokens
+            if aid >= 0:
+                t += wl.adapters[aid].n_trailer
+        assert t == P and not present[:P].all()
+        Q = orc.widen(wl.q[layer][0], s.dtype)
+        n = 0
+        for i in range(wl.q_len):
+            for h in range(s.n_q_heads):
+                hk = h // s.group
+                sc = (K[:P + i + 1, hk] @ Q[i, h]) / np.sqrt(s.head_dim)
+                sc = np.where(present[:P + i + 1, hk], sc, -np.inf)
+                w = np.exp(sc - sc.max())
+                o = (w[:, None] * V[:P + i + 1, hk]).sum(0) / w.sum()
+                assert np.max(np.abs(o - out[n])) <= 1e-12
+                assert abs(sc.max() + np.log(w.sum()) - lse[n]) <= 1e-12
+                n += 1
+
+
+def test_compressed_closed_forms():
+    wl = _compressed_case([0.4, 0.6, None], dtype="f32")
+    s = wl.shape
+    # constant values: the output is that constant whatever is pruned
+    for p in wl.packets:
+        p.v[...] = np.float32(0.75)
+    for a in wl.adapters:
+        a.hv[...] = np.float32(0.75)
+        a.tv[...] = np.float32(0.75)
+    wl.v_new[...] = np.float32(0.75)
+    out = oracle_outputs(wl, layer=0)[0][0]
+    assert np.max(np.abs(out - 0.75)) <= 1e-14
+    # a pruned key cannot matter: give it an enormous score and a wild value, nothing changes
+    wl2 = _compressed_case([0.4, 0.6, None])
+    ref = oracle_outputs(wl2, layer=0)[0][0]
+    p = wl2.packets[0]
+    dropped = sorted(set(range(p.n_tokens)) - set(int(x) for x in p.kept[0][0]))
+    assert dropped
+    p.k[0][dropped[0], 0, :] = np.float32(30.0)
+    p.v[0][dropped[0], 0, :] = np.float32(1e6)
+    got = oracle_outputs(wl2, layer=0)[0][0]
+    assert np.array_equal(got, ref)
