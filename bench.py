@@ -227,6 +227,51 @@ def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peak
     return res
 
 
+def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: float = 0.5):
+    """One layer of the config-3 shape (4 requests x 10 x 1024-token packets, 128 query tokens) with every
+    document pruned to about `keep` of its tokens, a different subset per kv head: attention kernel time,
+    and the rates counted on the keys that are actually held."""
+    import torch
+    from paper_2604_13226_b200 import binding as kvp, inputs as gen
+    from paper_2604_13226_b200.session import Session
+    shape = gen.ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
+    items = [[(10 * b + i, 0) for i in range(10)] for b in range(4)]
+    wl = gen.make_workload(shape, [1024] * 40, items, q_len=128, seed=seed, keep_rate=[keep] * 40)
+    sess = Session(wl, device=device)
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 1)
+    dev = torch.device(f"cuda:{device}")
+    sess.assemble()
+    qkv = sess.query_tensors(0)
+    att = []
+    for it in range(iters + 3):
+        flush_l2(torch, dev)
+        sess.prefill(0, qkv=qkv, want_lse=False)
+        torch.cuda.synchronize(dev)
+        a = sess.ctx.kernel_times(0)
+        if it >= 3:
+            att += a
+    assert sess.ctx.status_word() == 0
+    launch = sess.ctx.last_launch()
+    d, g, Lq = shape.head_dim, shape.group, 128
+    flops = bytes_ = 0.0
+    held = total = 0
+    for b in range(4):
+        for hk in range(shape.n_kv_heads):
+            keys = 10 * 32 + sum(len(wl.packets[pid].kept[0][hk]) for pid, _ in items[b])
+            held += keys - 320
+            total += 10 * 1024
+            flops += 4.0 * d * g * Lq * (keys + (Lq + 1) / 2.0)
+            bytes_ += 2.0 * d * 2 * keys
+    ms = statistics.median(att)
+    sess.close()
+    del sess, wl
+    torch.cuda.empty_cache()
+    return {"workload": "config3 shape, one layer, documents pruned per kv head", "kept_fraction": held / total, "attn_ms": ms,
+            "attn_tflops_on_held_keys": flops / ms / 1e9, "attn_gbs_on_held_keys": bytes_ / ms / 1e6,
+            "frac_tensor_sustained": flops / ms / 1e9 / peaks["bf16_tflops_sustained"], "launch": launch,
+            "l2": "flushed between iterations"}
+
+
 # ---------------------------------------------------------------------------------------------------
 # main
 # ---------------------------------------------------------------------------------------------------
@@ -424,6 +469,7 @@ def main():
                 extras["gather_materialise_point"] = measure_point("config5:16:64:1", args.seed, 10, True, peaks, local_rank)
                 # the step after the prefill: one new token per request over 16 x 33,280-token composed caches
                 extras["decode_point"] = measure_point("config5:16:1:16", args.seed, 10, False, peaks, local_rank)
+                extras["compressed_point"] = measure_compressed_point(args.seed, 10, peaks, local_rank)
             except Exception as ex:                                   # extras never invalidate the main line
                 extras["error"] = repr(ex)
             line["extra_points"] = extras
