@@ -73,6 +73,32 @@ def algorithmic_work(spec):
     return flops, bytes_
 
 
+# ---------------------------------------------------------------------------------------------------
+# multi-GPU: requests are sharded across ranks (every rank composes and prefills its own batch); the only
+# exchange is the barrier and the max-over-ranks of the timings
+# ---------------------------------------------------------------------------------------------------
+
+def rank_spec(workload: str, seed: int, rank: int):
+    """The batch rank `rank` works on: same shape, its own seeded draw of packets and requests (weak scaling)."""
+    return make_spec(workload, seed + 17 * rank)
+
+
+def max_over_ranks(values, world: int, device=None):
+    """Element-wise maximum of `values` (list of floats) over all ranks of the default process group."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_tokens_per_s(spec, world: int, ms_step: float) -> float:
+    """Whole-job rate: every rank pushes batch * q_len query tokens through the stack per step."""
+    return spec.batch * spec.q_len * world / (ms_step * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -344,7 +370,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    spec = make_spec(args.workload, args.seed + 17 * rank)         # weak scaling: every rank its own batch
+    spec = rank_spec(args.workload, args.seed, rank)               # weak scaling: every rank its own batch
     s = spec.shape
     wl = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
     sess = Session(wl, materialize=args.materialize, device=local_rank)
@@ -410,10 +436,7 @@ def main():
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, dev)
 
     sess.close()
     del sess
@@ -422,7 +445,7 @@ def main():
     if rank == 0:
         tokens = spec.batch * Lq * world
         ms_step = ms_total / args.steps
-        value = tokens / (ms_step * 1e-3)
+        value = job_tokens_per_s(spec, world, ms_step)
         flops, bytes_ = algorithmic_work(spec)
         a_ms = statistics.mean(attn_ms) if attn_ms else None
         tensor_bound = s.group * Lq >= 247

@@ -1,0 +1,61 @@
+"""The N > 1 path of the benchmark on CPU: two `gloo` ranks.  The path shards requests across ranks with no
+data-path collective (requests are independent, Section 3.2), so what there is to check is that every rank
+plans a different batch of the same shape, that the timing exchange takes the maximum over ranks, and that
+the whole-job rate counts every rank's tokens."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = r'''
+import json, os, sys
+sys.path.insert(0, os.environ["KVP_ROOT"])
+import torch.distributed as dist
+import bench
+from paper_2604_13226_b200 import binding as kvp
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", rank=rank, world_size=world)
+spec = bench.rank_spec("config5:3:16:2", 5, rank)
+s = spec.shape
+# host-only planning of this rank's batch through the C ABI: prefix lengths and the kernel's work list
+ctx = kvp.Context(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.dtype, rope_theta=s.rope_theta,
+                  max_packets=len(spec.packet_lens), max_adapters=1, max_batch=spec.batch,
+                  max_slots=sum(len(it) for it in spec.items), max_prefix_tokens=max(spec.prefix_len(b) for b in range(spec.batch)),
+                  max_query_tokens=spec.q_len, max_ws_rows=4096, device=-1)
+for n in spec.packet_lens:
+    ctx.register_packet(None, None, n, 0)
+ctx.register_adapter(None, None, spec.n_header, 0, None, None, spec.n_trailer, 0)
+aid, plen = ctx.assemble(spec.items, kvp.REBASE)
+cb, works, merges, n_slots = ctx.export_schedule(aid, spec.q_len)
+ms = bench.max_over_ranks([10.0 + rank, 7.0 - rank], world)
+dist.barrier()
+print(json.dumps({"rank": rank, "seed": spec.seed, "prefix": plen, "batch": spec.batch, "q_len": spec.q_len,
+                  "pieces": int(len(works)), "ms": ms, "value": bench.job_tokens_per_s(spec, world, ms[0])}))
+dist.destroy_process_group()
+'''
+
+
+def test_two_gloo_ranks_shard_requests_and_reduce_timings(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER)
+    port = 29500 + os.getpid() % 2000
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port),
+                   KVP_ROOT=ROOT, CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=240)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(json.loads(out.strip().splitlines()[-1]))
+    outs.sort(key=lambda d: d["rank"])
+    a, b = outs
+    assert a["seed"] != b["seed"]                                   # every rank draws its own batch
+    assert a["batch"] == b["batch"] == 2 and a["q_len"] == b["q_len"] == 16
+    assert a["prefix"] == b["prefix"] == [3 * (2048 + 32)] * 2      # same shape on every rank
+    assert a["pieces"] >= 1 and b["pieces"] >= 1
+    assert a["ms"] == b["ms"] == [11.0, 7.0]                        # maximum over ranks, element-wise
+    assert abs(a["value"] - 2 * 2 * 16 / 11.0e-3) < 1e-6 and a["value"] == b["value"]
