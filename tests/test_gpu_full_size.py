@@ -1,0 +1,128 @@
+"""GPU parity at the full sizes of the workloads the benchmark times (configs 3, 4 and points of the
+config-5 sweep), in the launch configuration `bench.py` uses (default tuning, documents read in place).
+The fp64 oracle cannot run gigabytes in seconds, so it computes sampled output rows one by one - fixed
+tokens {0, 1, 63, 64, 127, 128, last} plus seeded random (head, token) pairs - and every output row is
+additionally cross-checked between the tcgen05 kernel and the fp32 CUDA-core kernel.  The assembly's index
+map is compared bit for bit with the oracle's composition."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as orc
+from paper_2604_13226_b200 import binding as kvp
+from paper_2604_13226_b200 import inputs as gen
+from paper_2604_13226_b200.session import Session, torch_to_np
+from helpers import make_store, oracle_outputs
+
+pytestmark = pytest.mark.gpu
+
+BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
+
+
+def sample_rows(spec, seed, n_random=24):
+    s = spec.shape
+    rng = np.random.default_rng(seed)
+    toks = sorted(set([0, 1, 63, 64, 127, 128, spec.q_len - 1]) & set(range(spec.q_len)))
+    rows = {(int(rng.integers(s.n_q_heads)), t) for t in toks}
+    rows |= {(h, spec.q_len - 1) for h in range(0, s.n_q_heads, max(1, s.n_q_heads // 4))}
+    while len(rows) < len(toks) + 4 + n_random:
+        rows.add((int(rng.integers(s.n_q_heads)), int(rng.integers(spec.q_len))))
+    return sorted(rows)
+
+
+def check_sampled(wl, sess, layer, requests, seed):
+    spec, s = wl.spec, wl.shape
+    qkv = sess.query_tensors(layer)
+    out, lse = sess.prefill(layer, qkv=qkv)
+    assert sess.ctx.status_word() == 0 and sess.ctx.last_launch()["kind"] == 1
+    o = orc.widen(torch_to_np(out, s.dtype), s.dtype)
+    lse = lse.cpu().numpy().astype(np.float64)
+    rows = sample_rows(spec, seed)
+    st = make_store(wl)
+    f = orc.inv_freq(s.rope_theta, s.head_dim)
+    q, kn, vn = wl.query_layer(layer)
+    cs = wl.notes.get("chan_scale")
+    errs = []
+    for b in requests:
+        plan = orc.compose(st, wl.items[b], wl.rebase)
+        ro, rl, _, _ = orc.query_prefill(st, plan, layer, q[b], kn[b], vn[b], f, s.rope_pairing, rows=rows)
+        for n, (h, i) in enumerate(rows):
+            e = np.abs(o[b, i, h] - ro[n])
+            if cs is not None:
+                e = e / cs[layer, 0, h // s.group]
+            errs.append(e)
+            assert abs(lse[b, h, i] - rl[n]) <= 2e-2, (b, h, i)
+    errs = np.concatenate(errs)
+    assert errs.max() <= BF16_MAX_ABS and errs.mean() <= BF16_MEAN_ABS, (errs.max(), errs.mean())
+    return out, qkv
+
+
+def cross_check_all_rows(sess, layer, out, qkv):
+    ref, _ = sess.prefill(layer, kvp.FORCE_SIMPLE, qkv=qkv)
+    d = (out.float() - ref.float()).abs()
+    cs = sess.wl.notes.get("chan_scale")
+    if cs is not None:                     # a value channel multiplied by 8 carries 8x the rounding
+        g = sess.shape.group
+        d = d / torch.from_numpy(np.repeat(cs[layer, 0], g, axis=0)).to(d.device)[None, None]
+    assert float(d.max()) <= 3e-2 and float(d.mean()) <= 2e-3, (float(d.max()), float(d.mean()))
+
+
+def check_index_map(wl, sess, requests):
+    st = make_store(wl)
+    for b in requests:
+        plan = orc.compose(st, wl.items[b], wl.rebase)
+        src, dl, segs = sess.ctx.export_plan(sess.assembly_id, b)
+        assert np.array_equal(src, plan.src_row) and np.array_equal(dl, plan.delta) and np.array_equal(segs, plan.segments)
+
+
+def test_config3_full_size():
+    spec = gen.spec_config3(seed=0)
+    assert spec.shape.n_layers == 32 and spec.batch == 4 and spec.q_len == 128 and spec.prefix_len(0) == 10560
+    wl = gen.DeviceWorkload(spec, "cuda:0")
+    sess = Session(wl)
+    sess.assemble()
+    check_index_map(wl, sess, range(4))
+    for layer, reqs in ((0, [0, 3]), (17, [1]), (31, [2])):
+        out, qkv = check_sampled(wl, sess, layer, reqs, seed=100 + layer)
+    cross_check_all_rows(sess, 31, out, qkv)
+    sess.close()
+
+
+def test_config4_full_size_ragged_group7_outlier_channels():
+    spec = gen.spec_config4(seed=0)
+    s = spec.shape
+    assert (s.n_layers, s.n_q_heads, s.n_kv_heads) == (28, 28, 4) and spec.batch == 8 and spec.q_len == 256
+    assert len(set(spec.prefix_len(b) for b in range(8))) > 1                      # ragged prefixes
+    wl = gen.DeviceWorkload(spec, "cuda:0")
+    sess = Session(wl)
+    sess.assemble()
+    check_index_map(wl, sess, [0, 7])
+    shortest = min(range(8), key=spec.prefix_len)
+    longest = max(range(8), key=spec.prefix_len)
+    out, qkv = check_sampled(wl, sess, 0, [shortest], seed=200)
+    out, qkv = check_sampled(wl, sess, 27, [longest], seed=201)
+    cross_check_all_rows(sess, 27, out, qkv)
+    sess.close()
+
+
+@pytest.mark.parametrize("n_packets,q_len,batch,requests", [
+    (64, 16, 1, [0]),            # 133,120-token prefix, memory-bound
+    (2, 16, 16, [0, 15]),        # shortest prefix, widest batch
+    (16, 256, 4, [1]),           # compute-bound middle of the sweep
+    (64, 1024, 1, [0]),          # longest prefix x longest query
+    (64, 16, 16, [5]),           # the sweep's largest footprint: 1024 distinct packets, 8.6 GB of K/V
+    (8, 1, 4, [2]),              # a decode-sized query
+])
+def test_config5_sweep_points(n_packets, q_len, batch, requests):
+    spec = gen.spec_config5(n_packets, q_len, batch, seed=0)
+    assert spec.prefix_len(0) == n_packets * 2080
+    wl = gen.DeviceWorkload(spec, "cuda:0")
+    sess = Session(wl)
+    sess.assemble()
+    check_index_map(wl, sess, requests[:1])
+    out, qkv = check_sampled(wl, sess, 0, requests, seed=300 + n_packets + q_len)
+    if n_packets * q_len * batch <= 16 * 256 * 4:
+        cross_check_all_rows(sess, 0, out, qkv)
+    sess.close()
+    del sess, wl
+    torch.cuda.empty_cache()
