@@ -226,6 +226,26 @@ KVP_API int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q
                                     int32_t cta_cap, int32_t *works, int32_t work_cap, int32_t *merges,
                                     int32_t merge_cap, int32_t *counts);
 
+/*
+ * Attention mass per segment (the quantity behind the paper's attention maps, Section 4.4 / Fig. 5: how
+ * much of a query token's attention the header and trailer soft tokens of each packet absorb).  For query
+ * token i of request b and q head h:  mass[s] = sum over the keys j of segment s of exp(score_j - lse),
+ * with score_j = scale * q . R_Delta k_j (Eq. 1 applied to the cached key) and lse the value
+ * kvp_query_prefill returned for that row, so that the columns of a row add up to 1.
+ * Call it after kvp_query_prefill of the same layer with the same q, q_len and flags; the keys of the
+ * query block are the rows that call (and, with KVP_CONTINUE, the calls before it) appended.
+ *   q     device [batch][q_len][n_q_heads][head_dim]   (with KVP_ROPE_QUERY: ignored, the rotated copy
+ *                                                        the prefill made is used)
+ *   lse   device float [batch][n_q_heads][q_len]
+ *   mass  device float [batch][q_len][n_q_heads][n_cols]: column s < n_segments(b) is segment s of the
+ *         request in Eq. 2 order (header, document, trailer per slot; kvp_export_plan lists them), column
+ *         n_segments(b) the query block, further columns 0.  n_cols > largest n_segments.
+ * A diagnostic on CUDA cores, not part of the hot path.  Errors: INVALID, NOT_FOUND, STATE, CAPACITY
+ * (n_cols too small), CUDA.
+ */
+KVP_API int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const float *lse,
+                                 int32_t q_len, uint32_t flags, float *mass, int32_t n_cols, void *stream);
+
 /* Synchronises the device and returns the device-side status word (0 = no bounded wait ran out;
    otherwise a code identifying the wait) in *device_status, then clears it. */
 KVP_API int32_t kvp_status_word(kvp_ctx *ctx, int32_t *device_status);

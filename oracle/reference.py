@@ -283,6 +283,44 @@ def query_prefill(store: Store, plan: Plan, layer: int, q, k_new, v_new, inv_f: 
     return out, lse, K, V
 
 
+def segment_mass(store: Store, plan: Plan, layer: int, q, k_new, inv_f: np.ndarray, pairing: int = 0,
+                 scale: Optional[float] = None, rope_query: bool = False,
+                 rows: Optional[Sequence[Tuple[int, int]]] = None) -> np.ndarray:
+    """Attention mass per segment (Section 4.4, Fig. 5: what the attention maps show).  For each row
+    (head, query token i): softmax over the keys the token sees - the composed prefix (re-aligned by Eq. 1)
+    and query tokens <= i - then the probabilities are added up per segment of ``plan.segments`` and,
+    last column, over the query block.  Returns [n_rows][n_segments + 1]; every row sums to 1."""
+    Kp, _, _ = composed_kv(store, plan, layer, inv_f, pairing)
+    P = plan.prefix_len
+    Q = widen(q, store.dtype)
+    Kn = widen(k_new, store.dtype)
+    q_len, Hq, d = Q.shape
+    Hkv = Kp.shape[1]
+    g = Hq // Hkv
+    if rope_query:
+        pos = np.arange(P, P + q_len, dtype=np.int64)
+        Q = rope(Q, pos, inv_f, pairing)
+        Kn = rope(Kn, pos, inv_f, pairing)
+    if scale is None:
+        scale = 1.0 / np.sqrt(np.float64(d))
+    present = kept_mask(store, plan, layer, Hkv)
+    if rows is None:
+        rows = [(h, i) for i in range(q_len) for h in range(Hq)]
+    n_seg = plan.segments.shape[0]
+    out = np.zeros((len(rows), n_seg + 1), dtype=np.float64)
+    for n, (h, i) in enumerate(rows):
+        hk = h // g
+        sc = np.concatenate([Kp[:, hk] @ Q[i, h], Kn[:i + 1, hk] @ Q[i, h]]) * scale
+        if present is not None:
+            sc[:P][~present[:, hk]] = -np.inf
+        p = np.exp(sc - sc.max())
+        p /= p.sum()
+        for s_, (_, length, t0, _) in enumerate(plan.segments):
+            out[n, s_] = p[t0:t0 + length].sum()
+        out[n, n_seg] = p[P:].sum()
+    return out
+
+
 def kept_mask(store: Store, plan: Plan, layer: int, n_kv_heads: int):
     """present[t][h]: does kv head h of this layer still hold the key at composed position t?  None when
     the request has no compressed packet (everything is present)."""

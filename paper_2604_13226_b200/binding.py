@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         "kvp_export_plan": (i32, [vp, i32, i32, pi32, pi32, pi32, pi32]),
         "kvp_export_cache": (i32, [vp, i32, i32, i32, i32, vp, vp, i32, vp]),
         "kvp_export_schedule": (i32, [vp, i32, i32, pi32, i32, pi32, i32, pi32, i32, pi32]),
+        "kvp_segment_mass": (i32, [vp, i32, i32, vp, vp, i32, u32, vp, i32, vp]),
         "kvp_status_word": (i32, [vp, pi32]),
         "kvp_last_launch": (i32, [vp, pi32, pi32, pi32, pi32]),
         "kvp_tune": (i32, [vp, i32, i32]),
@@ -89,7 +90,7 @@ def lib() -> ctypes.CDLL:
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
-            "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_status_word", "kvp_last_launch", "kvp_tune",
+            "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_segment_mass", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
 
@@ -267,6 +268,14 @@ class Context:
                                                 works.ctypes.data_as(pi), works.shape[0],
                                                 merges.ctypes.data_as(pi), merges.shape[0], counts))
         return cb, works[:counts[1]], merges[:counts[2]], int(counts[3])
+
+    def segment_mass(self, assembly_id: int, layer: int, q, lse, q_len: int, n_cols: int, flags: int = 0, stream=None):
+        """float32 [batch][q_len][n_q_heads][n_cols] attention mass per segment (+ query block) of the last prefill."""
+        torch = self._torch
+        mass = torch.empty((q.shape[0], q_len, self.n_q_heads, n_cols), dtype=torch.float32, device=q.device)
+        self._check(self._L.kvp_segment_mass(self._h, assembly_id, layer, _ptr(q), _ptr(lse), q_len, flags, _ptr(mass),
+                                             n_cols, self._stream(stream)))
+        return mass
 
     def status_word(self) -> int:
         w = ctypes.c_int32(0)

@@ -964,6 +964,31 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     return KVP_OK;
 }
 
+int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const float *lse,
+                         int32_t q_len, uint32_t flags, float *mass, int32_t n_cols, void *stream)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "segment_mass: host-only context");
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "segment_mass: unknown assembly %d", assembly_id);
+    if (!q || !lse || !mass || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
+        return fail(ctx, KVP_ERR_INVALID, "segment_mass: bad arguments");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_CONTINUE | KVP_FORCE_SIMPLE)) return fail(ctx, KVP_ERR_INVALID, "segment_mass: unknown flags");
+    const kvp_assembly_host &as = ctx->slots[slot];
+    if (ctx->shape.group > 8) return fail(ctx, KVP_ERR_UNSUPPORTED, "segment_mass: more than 8 q heads per kv head");
+    if ((int)as.appended.size() != ctx->cfg.n_layers || as.appended[layer] < q_len)
+        return fail(ctx, KVP_ERR_STATE, "segment_mass: call kvp_query_prefill for this layer first");
+    if (as.flags & KVP_MATERIALIZE) return fail(ctx, KVP_ERR_UNSUPPORTED, "segment_mass: materialised assemblies keep no segment rows apart");
+    int max_seg = 0;
+    for (int b = 0; b < as.batch; ++b) max_seg = std::max(max_seg, as.items[b].seg_end - as.items[b].seg_begin);
+    if (n_cols <= max_seg) return fail(ctx, KVP_ERR_CAPACITY, "segment_mass: n_cols %d <= %d segments", n_cols, max_seg);
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const void *q_used = (flags & KVP_ROPE_QUERY) ? (const void *)ctx->q_scratch : q;
+    KVP_CUDA(ctx, kvp_launch_segment_mass(ctx->shape, plan_dev(ctx, slot), as.batch, q_len, as.appended[layer] - q_len, layer,
+                                          q_used, lse, ctx->pool_k, ctx->slot_k[slot], mass, n_cols, (cudaStream_t)stream));
+    return KVP_OK;
+}
+
 int32_t kvp_status_word(kvp_ctx *ctx, int32_t *device_status)
 {
     if (!ctx || !device_status) return KVP_ERR_INVALID;

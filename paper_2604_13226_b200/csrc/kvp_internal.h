@@ -184,6 +184,9 @@ cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int
                               int32_t prefix_len, int32_t n_query_rows, const char *pool_k, const char *pool_v,
                               const char *ws_k, const char *ws_v, void *k_out, void *v_out, int32_t k_as_f32,
                               cudaStream_t st);
+cudaError_t kvp_launch_segment_mass(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
+                                    int32_t q_pos0, int32_t layer, const void *q, const float *lse, const char *pool_k,
+                                    const char *ws_k, float *mass, int32_t n_cols, cudaStream_t st);
 cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
                                    int32_t q_pos0, int32_t layer, const void *q, const char *pool_k, const char *pool_v,
                                    const char *ws_k, const char *ws_v, void *out, float *lse, int32_t *ctas,

@@ -372,6 +372,83 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T 
     }
 }
 
+// ---- attention mass per segment (diagnostic) ----------------------------------------------------------
+// grid (batch * q_len, Hkv), 256 threads = 8 warps.  The block holds the group's q rows in fp32; each warp
+// takes every eighth key of a segment, each lane two rotation pairs of the key (Eq. 1 in fp32, as the
+// CUDA-core attention kernel does), scores by warp reduction, p = exp(scale * q.k' - lse) summed per head.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+segment_mass_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T *__restrict__ q,
+                    const float *__restrict__ lse, const char *__restrict__ pool_k, const char *__restrict__ ws_k,
+                    int64_t pool_rows, int64_t ws_rows, int n_q, int n_kv, int group, int pairing, float scale,
+                    float *__restrict__ mass, int n_cols)
+{
+    constexpr int HALF = D / 2, PPL = HALF / 32;            // rotation pairs per lane
+    extern __shared__ float sm[];                            // [group][D] q rows, [8][group] partial sums, [group] lse
+    float *qs = sm, *part = sm + group * D, *ls = part + 8 * group;
+    const int b = blockIdx.x / q_len, i = blockIdx.x % q_len, hk = blockIdx.y;
+    const kvp_item it = plan.items[layer * plan.item_stride + b];
+    const int plane = layer * n_kv + hk;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int w = threadIdx.x; w < group * D; w += blockDim.x)
+        qs[w] = Elem<T>::to_f32(q[(((int64_t)b * q_len + i) * n_q + hk * group + w / D) * D + w % D]);
+    for (int w = threadIdx.x; w < group; w += blockDim.x) ls[w] = lse[((int64_t)b * n_q + hk * group + w) * q_len + i];
+    __syncthreads();
+    float *out = mass + (((int64_t)b * q_len + i) * n_q + hk * group) * n_cols;
+    const int n_seg = it.seg_end - it.seg_begin;
+    for (int s = 0; s <= n_seg; ++s) {
+        // segment s, or (s == n_seg) the query block: appended rows 0 .. q_pos0 + i
+        const T *kb;
+        int n_keys, rope = 0;
+        if (s < n_seg) {
+            const kvp_seg sg = plan.segs[it.seg_begin + s];
+            kb = reinterpret_cast<const T *>(pool_k) + ((int64_t)plane * pool_rows + sg.src_row0) * D;
+            n_keys = sg.pad[2] >= 0 ? plan.kept[sg.pad[2] * plan.n_planes + plane] : sg.len;
+            rope = sg.rope;
+        } else {
+            kb = reinterpret_cast<const T *>(ws_k) + ((int64_t)plane * ws_rows + it.tail_row0) * D;
+            n_keys = q_pos0 + i + 1;
+        }
+        const float2 *cs = plan.rope + (size_t)rope * HALF;
+        float acc[8];
+#pragma unroll
+        for (int h = 0; h < 8; ++h) acc[h] = 0.f;
+        for (int j = warp; j < n_keys; j += 8) {
+            const T *kr = kb + (int64_t)j * D;
+            float ka[PPL], kc[PPL];
+            int ia[PPL], ib[PPL];
+#pragma unroll
+            for (int u = 0; u < PPL; ++u) {
+                const int pr = lane + 32 * u;
+                ia[u] = pairing ? 2 * pr : pr;
+                ib[u] = pairing ? 2 * pr + 1 : pr + HALF;
+                ka[u] = Elem<T>::to_f32(kr[ia[u]]);
+                kc[u] = Elem<T>::to_f32(kr[ib[u]]);
+                if (rope != 0) rotate_pair(ka[u], kc[u], cs[pr].x, cs[pr].y);
+            }
+            for (int h = 0; h < group; ++h) {
+                float d = 0.f;
+#pragma unroll
+                for (int u = 0; u < PPL; ++u) d += qs[h * D + ia[u]] * ka[u] + qs[h * D + ib[u]] * kc[u];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+                if (h < 8) acc[h] += expf(d * scale - ls[h]);
+            }
+        }
+        if (lane == 0)
+            for (int h = 0; h < group && h < 8; ++h) part[warp * group + h] = acc[h];
+        __syncthreads();
+        if (threadIdx.x < group) {
+            float t = 0.f;
+            for (int w = 0; w < 8; ++w) t += part[w * group + threadIdx.x];
+            out[(int64_t)threadIdx.x * n_cols + s] = t;
+        }
+        __syncthreads();
+    }
+    for (int w = threadIdx.x; w < group * (n_cols - n_seg - 1); w += blockDim.x)
+        out[(int64_t)(w / (n_cols - n_seg - 1)) * n_cols + n_seg + 1 + w % (n_cols - n_seg - 1)] = 0.f;
+}
+
 // ---- split-KV merge -----------------------------------------------------------------------------
 // Partials hold, per (unit, row): un-normalised O (fp32), the running max m of the raw scores and
 // the sum l of exp2((s - m) * c).  One block per (b, hk, m-tile, 16-row group), one thread per column.
@@ -472,6 +549,25 @@ cudaError_t kvp_launch_export(const kvp_shape &sh, const kvp_plan_dev &plan, int
         export_kernel<float><<<grid, 64, 0, st>>>(plan, b, layer, prefix_len, pool_k, pool_v, ws_k, ws_v, sh.pool_rows,
                                                  sh.ws_rows, sh.n_kv_heads, sh.head_dim, sh.pairing, k_out,
                                                  (float *)v_out, k_as_f32);
+    return cudaGetLastError();
+}
+
+cudaError_t kvp_launch_segment_mass(const kvp_shape &sh, const kvp_plan_dev &plan, int32_t batch, int32_t q_len,
+                                    int32_t q_pos0, int32_t layer, const void *q, const float *lse, const char *pool_k,
+                                    const char *ws_k, float *mass, int32_t n_cols, cudaStream_t st)
+{
+    const dim3 grid(batch * q_len, sh.n_kv_heads);
+    const size_t smem = sizeof(float) * ((size_t)sh.group * sh.head_dim + 9 * sh.group);
+#define KVP_MASS(T, D)                                                                                              \
+    segment_mass_kernel<T, D><<<grid, 256, smem, st>>>(plan, q_len, q_pos0, layer, (const T *)q, lse, pool_k, ws_k,  \
+                                                       sh.pool_rows, sh.ws_rows, sh.n_q_heads, sh.n_kv_heads,       \
+                                                       sh.group, sh.pairing, sh.scale, mass, n_cols)
+    if (sh.dtype == KVP_DTYPE_BF16) {
+        if (sh.head_dim == 128) KVP_MASS(__nv_bfloat16, 128); else KVP_MASS(__nv_bfloat16, 64);
+    } else {
+        if (sh.head_dim == 128) KVP_MASS(float, 128); else KVP_MASS(float, 64);
+    }
+#undef KVP_MASS
     return cudaGetLastError();
 }
 

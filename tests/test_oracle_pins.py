@@ -10,7 +10,7 @@ import pytest
 from oracle import bruteforce as bf
 from oracle import reference as orc
 from paper_2604_13226_b200 import inputs as gen
-from helpers import oracle_outputs
+from helpers import make_store, oracle_outputs
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -409,3 +409,39 @@ def test_compressed_closed_forms():
     p.v[0][dropped[0], 0, :] = np.float32(1e6)
     got = oracle_outputs(wl2, layer=0)[0][0]
     assert np.array_equal(got, ref)
+
+
+# ------------------------------------------------------------------------------------------------
+# attention mass per segment
+# ------------------------------------------------------------------------------------------------
+
+def test_segment_mass_rows_sum_to_one_and_match_closed_forms():
+    shape = gen.ModelShape(1, 4, 2, 64, "f32", 10000.0, 0)
+    wl = gen.make_workload(shape, [50, 33], [[(0, 0), (1, -1)]], q_len=5, n_header=3, n_trailer=2, seed=3)
+    st = make_store(wl)
+    plan = orc.compose(st, wl.items[0])
+    f = orc.inv_freq(shape.rope_theta, 64)
+    m = orc.segment_mass(st, plan, 0, wl.q[0][0], wl.k_new[0][0], f)
+    assert m.shape == (5 * 4, 4 + 1) and np.max(np.abs(m.sum(1) - 1.0)) <= 1e-14 and m.min() >= 0
+    # consistency with the attention routine: exp(score - lse) summed over everything is the same 1,
+    # and with V replaced by one-hot segment indicators the attention output IS the mass
+    P = plan.prefix_len
+    ind = np.zeros((P + 5, 2, 64))
+    for s_, (_, length, t0, _) in enumerate(plan.segments):
+        ind[t0:t0 + length, :, s_] = 1.0
+    ind[P:, :, 4] = 1.0
+    Kp, _, _ = orc.composed_kv(st, plan, 0, f)
+    K = np.concatenate([Kp, orc.widen(wl.k_new[0][0], "f32")])
+    o, _ = orc.attention_rows(K, ind, orc.widen(wl.q[0][0], "f32"), P, 1.0 / 8.0)
+    assert np.max(np.abs(o[:, :5] - m)) <= 1e-14
+    # all keys equal: every visible key gets the same probability, mass = segment length / keys seen
+    for p in wl.packets:
+        p.k[...] = np.float32(0.25)
+    for a in wl.adapters:
+        a.hk[...] = np.float32(0.25)
+        a.tk[...] = np.float32(0.25)
+    wl.k_new[...] = np.float32(0.25)
+    plan0 = orc.compose(st, wl.items[0], rebase=False)
+    m = orc.segment_mass(st, plan0, 0, wl.q[0][0], wl.k_new[0][0], f, rows=[(1, 2)])
+    seen = P + 3
+    assert np.allclose(m[0], [3 / seen, 50 / seen, 2 / seen, 33 / seen, 3 / seen], atol=1e-14)
