@@ -199,6 +199,11 @@ def composed_kv(store: Store, plan: Plan, layer: int, inv_f: np.ndarray, pairing
         assert k.shape[0] == n and v.shape[0] == n
         ks.append(widen(k, store.dtype))
         vs.append(widen(v, store.dtype))
+    if not ks:
+        # a request without packets: the concatenation of Eq. 2 over zero slots is the empty sequence
+        like = store.packets[0][1](layer)[0] if store.packets else store.adapters[0][2](layer)[0]
+        empty = np.zeros((0,) + tuple(like.shape[1:]), dtype=np.float64)
+        return empty, empty.copy(), empty.copy()
     k_raw = np.concatenate(ks, axis=0)
     v_cat = np.concatenate(vs, axis=0)
     k_reb = rope(k_raw, plan.delta.astype(np.int64), inv_f, pairing)

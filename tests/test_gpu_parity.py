@@ -7,6 +7,7 @@ the workload multiplies by 8 ("outlier channel") carries 8x the value, 8x the bf
 output and of the probabilities, and therefore 8x the bound."""
 import numpy as np
 import pytest
+import torch
 
 from oracle import reference as orc
 from paper_2604_13226_b200 import binding as kvp
@@ -262,4 +263,34 @@ def test_short_query_many_splits_and_tensor_vs_simple_kernel():
     a, _ = sess.prefill(0)
     b, _ = sess.prefill(0, kvp.FORCE_SIMPLE)
     assert float((a.float() - b.float()).abs().max()) <= 2e-2
+    sess.close()
+
+
+def test_empty_request_in_a_batch_and_lone_query_token():
+    # a request with no packets at all (prefix length 0) next to a normal one: its query tokens attend to
+    # the query block only; with one token the output is that token's own value row
+    shape = gen.ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
+    wl = gen.make_workload(shape, [300], [[], [(0, 0)]], q_len=1, seed=12)
+    sess = Session(wl)
+    aid, plen = sess.assemble()
+    assert plen == [0, 332]
+    out, lse = sess.prefill(0)
+    assert sess.ctx.status_word() == 0
+    o = out.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(o[0, 0], np.repeat(wl.v_new[0][0, 0], shape.group, axis=0))       # softmax over one key
+    check_attention(wl, sess)
+    sess.close()
+    wl = gen.make_workload(shape, [300], [[], [(0, 0)]], q_len=70, seed=13)
+    sess = Session(wl)
+    sess.assemble()
+    check_attention(wl, sess)
+    sess.close()
+
+
+def test_bf16_head_dim_64_uses_the_cuda_core_kernel():
+    wl = ragged_small("bf16", 64)
+    sess = Session(wl)
+    sess.assemble()
+    check_attention(wl, sess)
+    assert sess.ctx.last_launch()["kind"] == 0
     sess.close()

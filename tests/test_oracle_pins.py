@@ -445,3 +445,18 @@ def test_segment_mass_rows_sum_to_one_and_match_closed_forms():
     m = orc.segment_mass(st, plan0, 0, wl.q[0][0], wl.k_new[0][0], f, rows=[(1, 2)])
     seen = P + 3
     assert np.allclose(m[0], [3 / seen, 50 / seen, 2 / seen, 33 / seen, 3 / seen], atol=1e-14)
+
+
+def test_empty_prefix_is_plain_causal_attention_over_the_query_block():
+    shape = gen.ModelShape(1, 4, 2, 64, "f32", 10000.0, 0)
+    wl = gen.make_workload(shape, [20], [[]], q_len=6, seed=4)
+    out, lse, K, V, plan = oracle_outputs(wl)[0]
+    assert plan.prefix_len == 0 and K.shape[0] == 6
+    Q = orc.widen(wl.q[0][0], "f32")
+    n = 0
+    for i in range(6):
+        for h in range(4):
+            sc = (K[:i + 1, h // 2] @ Q[i, h]) / 8.0
+            w = np.exp(sc - sc.max())
+            assert np.max(np.abs((w[:, None] * V[:i + 1, h // 2]).sum(0) / w.sum() - out[n])) <= 1e-14
+            n += 1
