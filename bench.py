@@ -312,6 +312,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the extra roofline points and the CPU baseline")
     ap.add_argument("--materialize", action="store_true", help="materialise the composed prefix instead of reading in place")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time the attention kernel over the config-5 grid (packets x q_len x batch) and print one JSON line per point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -322,6 +324,19 @@ def main():
 
     import torch
     from paper_2604_13226_b200 import inputs as gen
+
+    if args.sweep:
+        if rank != 0:
+            return
+        assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+        for n in (2, 4, 8, 16, 32, 64):
+            for ql in (16, 64, 256, 1024):
+                for b in (1, 4, 16):
+                    r = measure_point(f"config5:{n}:{ql}:{b}", args.seed, 5, False, peaks, local_rank)
+                    r.pop("gather_ms", None); r.pop("gather_gbs", None); r.pop("gather_frac_hbm", None); r.pop("gather_bytes", None)
+                    r.update({"packets": n, "q_len": ql, "batch": b, "bound": "tensor" if 4 * ql >= 247 else "hbm"})
+                    print(json.dumps(r), flush=True)
+        return
 
     if args.impl == "reference":
         if rank != 0:
