@@ -141,6 +141,19 @@ bool make_tensor_map(encode_tiled_fn enc, CUtensorMap *tm, void *base, int head_
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The caller's k_new or v_new, [batch][q_len][Hkv][d] bf16, as a 4-D tensor (d, Hkv, q_len, batch); box = 64
+// columns x 1 head x 128 tokens, the same shared-memory tile as a pool box.  Tokens past q_len read as zero.
+bool make_query_tensor_map(encode_tiled_fn enc, CUtensorMap *tm, const void *base, int head_dim, int n_kv, int q_len, int batch)
+{
+    const cuuint64_t dims[4] = {(cuuint64_t)head_dim, (cuuint64_t)n_kv, (cuuint64_t)q_len, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_kv * head_dim * 2, (cuuint64_t)q_len * n_kv * head_dim * 2};
+    const cuuint32_t box[4] = {64, 1, KVP_TILE_KEYS, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr int kMaxTimed = 4096;
 
 // Record an event before (edge 0) / after (edge 1) a timed kernel; events are created on first use.
@@ -480,6 +493,7 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess && fn &&
             qres == cudaDriverEntryPointSuccess) {
             encode_tiled_fn enc = (encode_tiled_fn)fn;
+            ctx->encode_tiled = fn;
             const int planes = sh.n_layers * sh.n_kv_heads;
             bool ok = make_tensor_map(enc, &ctx->tm_pool_k, ctx->pool_k, sh.head_dim, sh.pool_rows, planes) &&
                       make_tensor_map(enc, &ctx->tm_pool_v, ctx->pool_v, sh.head_dim, sh.pool_rows, planes);
@@ -867,14 +881,24 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     const double *inv_freq_dev = reinterpret_cast<const double *>((char *)ctx->cfg.workspace + 256);
 
     int launches = 0;
-    KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q_pos0, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
-                                    layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
-    ++launches;
+    const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
+    // plain prefill on the two-stream kernel: it reads the query block's K/V from k_new / v_new and appends them itself
+    kvp_attn2_args a;
+    a.tail_direct = 0;
+    if (fast && ctx->kernel_variant == 0 && ctx->fused_append && !rope_query && q_pos0 == 0 &&
+        (((uintptr_t)k_new | (uintptr_t)v_new) & 15) == 0 &&
+        make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_knew, k_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch) &&
+        make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_vnew, v_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch))
+        a.tail_direct = 1;
+    if (!a.tail_direct) {
+        KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q_pos0, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
+                                        layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
+        ++launches;
+    }
     const void *q_used = rope_query ? (const void *)ctx->q_scratch : q;
     as.last_q_len = q_len;
     as.appended[layer] = q_pos0 + q_len;
 
-    const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
     int32_t ctas = 0, splits = 1;
     if (!fast) {
         KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
@@ -892,7 +916,10 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         }
         const kvp_assembly_host::sched_state &ss = as.sched[li];
         const char *sd = ctx->slot_sched_dev[slot] + ctx->sched_bytes * li;
-        kvp_attn2_args a;
+        a.k_new = k_new;
+        a.v_new = v_new;
+        a.ws_k = ctx->slot_k[slot];
+        a.ws_v = ctx->slot_v[slot];
         a.plan = plan;
         a.q_len = q_len;
         a.q_pos0 = q_pos0;
@@ -1056,6 +1083,7 @@ int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
         (key == KVP_TUNE_SPLIT_TARGET_CTAS ? ctx->split_target_ctas : ctx->force_splits) = value;
         for (kvp_assembly_host &as : ctx->slots) as.sched.clear();       // work lists are rebuilt on next use
     }
+    else if (key == KVP_TUNE_FUSED_APPEND) ctx->fused_append = value != 0;
     else if (key == KVP_TUNE_KERNEL_VARIANT) {
         if (value != 0 && value != 1) return fail(ctx, KVP_ERR_INVALID, "tune: kernel variant %d", value);
         ctx->kernel_variant = value;

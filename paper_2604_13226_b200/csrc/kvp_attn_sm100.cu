@@ -66,6 +66,12 @@ struct Params {
     float *partial_o;
     float2 *partial_ml;
     int32_t *status;
+    // tail_direct: the query block's tiles come from k_new / v_new ([batch][q_len][Hkv][d], through their own
+    // tensor maps) and the kernel copies those rows into the workspace rows (the append) itself
+    int tail_direct;
+    const uint4 *k_new, *v_new;
+    uint4 *ws_k, *ws_v;
+    long long ws_rows;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
@@ -134,6 +140,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, int w, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
         : "memory");
 }
 
@@ -297,9 +311,9 @@ __device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
 {
     Tile t;
     if (j < w.n_tail) {
-        t.row0 = w.tail_row0 + j * KVP_TILE_KEYS;
+        t.row0 = p.tail_direct ? j * KVP_TILE_KEYS : w.tail_row0 + j * KVP_TILE_KEYS;
         t.n_keys = min(KVP_TILE_KEYS, p.q_pos0 + p.q_len - j * KVP_TILE_KEYS);
-        t.src = 1;
+        t.src = p.tail_direct ? 2 : 1;               // 2: rows of the caller's k_new / v_new, by query token
         t.rope = 0;
         t.qoff = j * KVP_TILE_KEYS;
     } else {
@@ -656,6 +670,18 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
         const int n_rows = p.group * p.q_len;
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
+        if (p.tail_direct && w.lo == 0 && w.row_base == 0) {
+            // the piece that starts a (request, kv head) appends the query block's K/V rows behind the prefix
+            for (int i = t; i < p.q_len; i += 128) {
+                const long long srow = (((long long)w.b * p.q_len + i) * p.n_kv + w.hk) * 16;
+                const long long drow = ((long long)w.plane * p.ws_rows + w.tail_row0 + i) * 16;
+#pragma unroll 4
+                for (int c4 = 0; c4 < 16; ++c4) {
+                    p.ws_k[drow + c4] = __ldg(p.k_new + srow + c4);
+                    p.ws_v[drow + c4] = __ldg(p.v_new + srow + c4);
+                }
+            }
+        }
         auto produce = [&](int s, int rope, uint32_t &nEp) {
             const int buf = nEp & 1;
             if (nEp >= 2) {                                 // the epoch before last used this buffer
@@ -690,7 +716,8 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
 // ---- TMA producer (whole warp; lane 0 issues) ----------------------------------------------------------
 __device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const int lane, const CUtensorMap *tm_pool_k,
                                          const CUtensorMap *tm_pool_v, const CUtensorMap *tm_ws_k,
-                                         const CUtensorMap *tm_ws_v)
+                                         const CUtensorMap *tm_ws_v, const CUtensorMap *tm_knew,
+                                         const CUtensorMap *tm_vnew)
 {
     uint32_t ring_n = 0;                                   // loads issued before this piece
     bool ok = true;
@@ -722,11 +749,17 @@ __device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const in
                     const uint32_t stage = g % kStages, use = g / kStages;
                     if (use > 0) ok = mbar_wait(c.bar(kKvEmpty + stage), (use - 1) & 1, c.abort_flag, p.status, 10 + stage);
                     if (ok) {
-                        const CUtensorMap *tm = src_i == 0 ? (kv_i ? tm_pool_v : tm_pool_k) : (kv_i ? tm_ws_v : tm_ws_k);
                         const uint32_t dst = c.smem_base + kOffRing + stage * kTileBytes;
                         mbar_expect_tx(c.bar(kKvFull + stage), kTileBytes);
-                        tma_load_3d(dst, tm, 0, row0_i, w.plane, c.bar(kKvFull + stage));
-                        tma_load_3d(dst + kHalfBytes, tm, 64, row0_i, w.plane, c.bar(kKvFull + stage));
+                        if (src_i == 2) {
+                            const CUtensorMap *tm = kv_i ? tm_vnew : tm_knew;
+                            tma_load_4d(dst, tm, 0, w.hk, row0_i, w.b, c.bar(kKvFull + stage));
+                            tma_load_4d(dst + kHalfBytes, tm, 64, w.hk, row0_i, w.b, c.bar(kKvFull + stage));
+                        } else {
+                            const CUtensorMap *tm = src_i == 0 ? (kv_i ? tm_pool_v : tm_pool_k) : (kv_i ? tm_ws_v : tm_ws_k);
+                            tma_load_3d(dst, tm, 0, row0_i, w.plane, c.bar(kKvFull + stage));
+                            tma_load_3d(dst + kHalfBytes, tm, 64, row0_i, w.plane, c.bar(kKvFull + stage));
+                        }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -856,6 +889,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_constant__ CUtensorMap tm_pool_v,
                   const __grid_constant__ CUtensorMap tm_ws_k, const __grid_constant__ CUtensorMap tm_ws_v,
+                  const __grid_constant__ CUtensorMap tm_knew, const __grid_constant__ CUtensorMap tm_vnew,
                   const Params p)
 {
     extern __shared__ char smem_raw[];
@@ -910,7 +944,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
         if (warp == 12) {
             mma_role(p, c);
         } else if (warp == 13) {
-            tma_role(p, c, lane, &tm_pool_k, &tm_pool_v, &tm_ws_k, &tm_ws_v);
+            tma_role(p, c, lane, &tm_pool_k, &tm_pool_v, &tm_ws_k, &tm_ws_v, &tm_knew, &tm_vnew);
         }
     }
 
@@ -1019,7 +1053,16 @@ cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, 
     p.partial_o = a.partial_o;
     p.partial_ml = a.partial_ml;
     p.status = a.status;
-    attn_sm100_kernel<<<a.n_ctas, kThreads, kSmemBytes, st>>>(tm_pool_k, tm_pool_v, tm_ws_k, tm_ws_v, p);
+    p.tail_direct = a.tail_direct;
+    p.k_new = (const uint4 *)a.k_new;
+    p.v_new = (const uint4 *)a.v_new;
+    p.ws_k = (uint4 *)a.ws_k;
+    p.ws_v = (uint4 *)a.ws_v;
+    p.ws_rows = sh.ws_rows;
+    // without tail_direct the two query maps are never dereferenced: any valid map will do
+    attn_sm100_kernel<<<a.n_ctas, kThreads, kSmemBytes, st>>>(tm_pool_k, tm_pool_v, tm_ws_k, tm_ws_v,
+                                                              a.tail_direct ? a.tm_knew : tm_ws_k,
+                                                              a.tail_direct ? a.tm_vnew : tm_ws_v, p);
     return cudaGetLastError();
 }
 

@@ -144,6 +144,8 @@ struct kvp_ctx {
     uint64_t sched_off_works = 0, sched_off_merges = 0, sched_bytes = 0;
     int32_t sched_max_works = 0, sched_max_merges = 0;
     int32_t kernel_variant = 0;            // 0: two-stream kernel, 1: single-tile kernel
+    int32_t fused_append = 1;              // plain prefill: the attention kernel reads k_new / v_new itself and appends them
+    void *encode_tiled = nullptr;          // cuTensorMapEncodeTiled
     float *partial_o = nullptr;            // [units][128][head_dim]
     float2 *partial_ml = nullptr;          // [units][128] (running max, running sum)
     char *q_scratch = nullptr;
@@ -221,6 +223,12 @@ struct kvp_attn2_args {
     float *partial_o;
     float2 *partial_ml;
     int32_t *status;
+    // tail_direct: the query block's K/V tiles are loaded from k_new / v_new ([batch][q_len][Hkv][d]) through
+    // tm_knew / tm_vnew and the kernel copies those rows into the workspace rows itself
+    int32_t tail_direct;
+    const void *k_new, *v_new;
+    char *ws_k, *ws_v;
+    CUtensorMap tm_knew, tm_vnew;
 };
 cudaError_t kvp_attn_sm100_prepare(void);
 cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, const CUtensorMap &tm_pool_k,

@@ -177,7 +177,24 @@ def test_config2_cta_counts(ctas, no_split):
     ll = sess.ctx.last_launch()
     assert ll["kind"] == 1 and ll["ctas"] <= ctas
     if no_split:
-        assert ll["splits"] == 1 and ll["launches"] == 2
+        assert ll["splits"] == 1 and ll["launches"] == 1     # the attention kernel appends the query block itself
+    sess.close()
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_config2_append_fused_or_separate(fused):
+    # the query block's K/V reach the cache either through the attention kernel's own copy or the append kernel:
+    # same attention output, same appended rows
+    wl = gen.config2()
+    sess = Session(wl)
+    sess.assemble()
+    sess.ctx.tune(kvp.TUNE_FUSED_APPEND, fused)
+    check_attention(wl, sess)
+    assert sess.ctx.last_launch()["launches"] == (1 if fused else 2) + (sess.ctx.last_launch()["splits"] > 1)
+    for b in range(len(wl.items)):
+        k, v = sess.ctx.export_cache(sess.assembly_id, 0, b, sess.prefix_len[b], wl.q_len)
+        assert np.array_equal(torch_to_np(k, "bf16")[sess.prefix_len[b]:], wl.k_new[0][b])
+        assert np.array_equal(torch_to_np(v, "bf16")[sess.prefix_len[b]:], wl.v_new[0][b])
     sess.close()
 
 
