@@ -831,8 +831,114 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
         if (k + 2 < n_steps) ms.nxt = get_tile(p, wq, stream_tile(wq, s, k + 2));
     };
 
+    // ---- a piece in mode 0: both streams take every tile; loads arrive K(0) V(0) K(1) V(1) ... -----------------
+    // This is the tensor-bound path, and the issuing warp's own instruction time is what bounds it, so
+    // the loop is kept short: tile facts (key count, document) are fetched 32 tiles at a time, one per
+    // lane, and handed round by shuffle; ring stages advance incrementally; all waits of a block come
+    // first, with one vote and one fence.
+    const int lane = threadIdx.x & 31;
+    auto piece_mode0 = [&](const Work &w) {
+        const int n = w.n;
+        uint32_t stK = ring_n % kStages, parK = (ring_n / kStages) & 1;                 // K(k), used at step k
+        uint32_t stV = (ring_n + 1) % kStages, parV = ((ring_n + 1) / kStages) & 1;     // V(k - 1), used at step k
+        auto advance = [](uint32_t &st_, uint32_t &par_) {                              // two loads further on
+            if (st_ == 0) st_ = 2; else { st_ -= 1; par_ ^= 1; }
+        };
+        int b0 = 0, nk_l = 0, rope_l = 0;
+        auto refill = [&](int from) {
+            b0 = from;
+            if (from + lane < n) {
+                const Tile t = get_tile(p, w, w.lo + from + lane);
+                nk_l = t.n_keys;
+                rope_l = t.rope;
+            }
+        };
+        refill(0);
+        int prev_nk = 0, prev_rope = 0;
+        for (int k = 0; k <= n && ok; ++k) {
+            if (k - b0 == 31) refill(k);                          // tile k + 1 stays inside the batch
+            const int nk = __shfl_sync(0xffffffffu, nk_l, k - b0);
+            const int rope = __shfl_sync(0xffffffffu, rope_l, k - b0);
+            const int rope_n = __shfl_sync(0xffffffffu, rope_l, (k + 1 - b0) & 31);
+            const bool newq = (k == 0) || rope != prev_rope;      // first tile of a document: its own Q buffer
+            const bool lastq = (k + 1 >= n) || rope_n != rope;
+            auto step = [&](auto s_c) {
+                constexpr int s = decltype(s_c)::value;
+                MmaStream &ms = st[s];
+                // ---- waits of the block ---------------------------------------------------------
+                if (k >= 1) {
+                    if (s == 0) ok = mbar_wait(c.bar(kKvFull + stV), parV, c.abort_flag, p.status, 23);
+                    if (ok) ok = mbar_wait(c.bar(kPFull + s), ms.nP & 1, c.abort_flag, p.status, 24 + s);
+                    ++ms.nP;
+                    if (ok && k == 1 && ms.nItems > 0)
+                        ok = mbar_wait(c.bar(kOFree + s), (ms.nItems - 1) & 1, c.abort_flag, p.status, 26 + s);
+                }
+                if (k < n) {
+                    if (newq) {
+                        ms.qbuf = ms.nEpoch & 1;
+                        if (ok) ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
+                        ++ms.nEpoch;
+                    }
+                    if (s == 0 && ok) ok = mbar_wait(c.bar(kKvFull + stK), parK, c.abort_flag, p.status, 22);
+                }
+                ok = __all_sync(0xffffffffu, ok);                 // the lanes stay together
+                if (!ok) return;
+                tc_fence_after();
+                if (k >= 1) {
+                    // ---- O_s += P_s V of step k-1 ---------------------------------------------------
+                    const uint32_t v_lo = desc_lo(c.smem_base + kOffRing + stV * kTileBytes, kHalfBytes);
+                    const uint32_t pa = c.tmem + kColS + s * 128;
+                    const uint32_t oa = c.tmem + kColO + s * 128;
+                    if (prev_nk == KVP_TILE_KEYS && k > 1) {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)           // 16 keys per step: P advances 8 columns, V 2048 bytes
+                            mma_ts_c<1>(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv);
+                    } else {
+                        const int ksteps = max(1, (prev_nk + 15) >> 4);    // an empty tile still initialises O (P = 0)
+                        for (int kk = 0; kk < ksteps; ++kk)
+                            mma_ts(oa, pa + kk * 8, desc64(v_lo + kk * 128, kDescHi), idesc_pv, (k > 1 || kk > 0));
+                    }
+                    if (s == 1) tc_commit(c.bar(kKvEmpty + stV));
+                    if (k == n) {
+                        tc_commit(c.bar(kOFull + s));
+                        ++ms.nItems;
+                    }
+                }
+                if (k < n) {
+                    // ---- S_s = Q_s K^T of step k ----------------------------------------------------
+                    const uint32_t n16 = max(16u, (uint32_t)(nk + 15) & ~15u);         // a tile may be empty for this head
+                    const uint32_t idesc = instr_desc(n16, 0);
+                    const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
+                    const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stK * kTileBytes, 16);
+                    const uint32_t d = c.tmem + kColS + s * 128;
+                    mma_ss<0>(d, desc64(q_lo, kDescHi), desc64(k_lo, kDescHi), idesc);
+#pragma unroll
+                    for (int kk = 1; kk < 8; ++kk) {             // 16 columns per step: 32 bytes, second half 16 KB on
+                        constexpr uint32_t kHalf16 = kHalfBytes >> 4;
+                        const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
+                        mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+                    }
+                    tc_commit(c.bar(kSFull + s));
+                    if (s == 1) tc_commit(c.bar(kKvEmpty + stK));
+                    if (lastq) tc_commit(c.bar(kQFree + 2 * s + ms.qbuf));
+                }
+            };
+            step(std::integral_constant<int, 0>{});
+            if (ok) step(std::integral_constant<int, 1>{});
+            if (k >= 1) advance(stV, parV);
+            if (k < n) advance(stK, parK);
+            prev_nk = nk;
+            prev_rope = rope;
+        }
+    };
+
     for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
         const Work w = load_work(p, wi);
+        if (w.mode == 0) {
+            piece_mode0(w);
+            ring_n += 2u * (uint32_t)w.n;
+            continue;
+        }
         const int steps[2] = {w.steps0, w.steps1};
         const int max_steps = max(w.steps0, w.steps1);
         auto block = [&](auto s_c, int k) {
