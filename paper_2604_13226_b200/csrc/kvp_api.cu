@@ -217,11 +217,14 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     std::vector<unit_t> units;
     const int n_rows = sh.group * q_len;
     int64_t total = 0;
-    for (int b = 0; b < as.batch; ++b) {
-        const kvp_item &item = as.items[(as.item_stride ? layer * as.item_stride : 0) + b];
-        const int n_prefix = item.tile_end - item.tile_begin;
-        for (int hk = 0; hk < sh.n_kv_heads; ++hk)
-            for (int row_base = 0; row_base < n_rows; row_base += 2 * KVP_TILE_ROWS) {
+    // Row blocks outermost: the units of one (request, kv head) - which stream the same K/V - then lie a
+    // whole number of CTA shares apart on the line (when their count divides the CTA count), so the CTAs
+    // that hold them reach the same key tiles at the same time and all but the first find them in L2.
+    for (int row_base = 0; row_base < n_rows; row_base += 2 * KVP_TILE_ROWS)
+        for (int b = 0; b < as.batch; ++b) {
+            const kvp_item &item = as.items[(as.item_stride ? layer * as.item_stride : 0) + b];
+            const int n_prefix = item.tile_end - item.tile_begin;
+            for (int hk = 0; hk < sh.n_kv_heads; ++hk) {
                 unit_t u;
                 u.b = b; u.hk = hk; u.row_base = row_base;
                 u.mode = (n_rows - row_base <= KVP_TILE_ROWS) ? 1 : 0;
@@ -231,7 +234,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 units.push_back(u);
                 total += (int64_t)u.n_all * (u.mode ? 1 : 2) + kPieceCost;
             }
-    }
+        }
     int G = std::min(ctx->sm_count, kMaxCtas);
     if (ctx->split_target_ctas > 0) G = std::min(ctx->split_target_ctas, kMaxCtas);
     const bool no_split = ctx->force_splits == 1;               // cuts only between units

@@ -866,8 +866,11 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 constexpr int s = decltype(s_c)::value;
                 MmaStream &ms = st[s];
                 // ---- waits of the block ---------------------------------------------------------
+                if (s == 0) {                                 // the tiles first: they land while P is being formed
+                    if (k >= 1) ok = mbar_wait(c.bar(kKvFull + stV), parV, c.abort_flag, p.status, 23);
+                    if (k < n && ok) ok = mbar_wait(c.bar(kKvFull + stK), parK, c.abort_flag, p.status, 22);
+                }
                 if (k >= 1) {
-                    if (s == 0) ok = mbar_wait(c.bar(kKvFull + stV), parV, c.abort_flag, p.status, 23);
                     if (ok) ok = mbar_wait(c.bar(kPFull + s), ms.nP & 1, c.abort_flag, p.status, 24 + s);
                     ++ms.nP;
                     if (ok && k == 1 && ms.nItems > 0)
@@ -879,7 +882,6 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                         if (ok) ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
                         ++ms.nEpoch;
                     }
-                    if (s == 0 && ok) ok = mbar_wait(c.bar(kKvFull + stK), parK, c.abort_flag, p.status, 22);
                 }
                 ok = __all_sync(0xffffffffu, ok);                 // the lanes stay together
                 if (!ok) return;
