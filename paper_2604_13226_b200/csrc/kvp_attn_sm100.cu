@@ -670,18 +670,6 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
         const int n_rows = p.group * p.q_len;
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
-        if (p.tail_direct && w.lo == 0 && w.row_base == 0) {
-            // the piece that starts a (request, kv head) appends the query block's K/V rows behind the prefix
-            for (int i = t; i < p.q_len; i += 128) {
-                const long long srow = (((long long)w.b * p.q_len + i) * p.n_kv + w.hk) * 16;
-                const long long drow = ((long long)w.plane * p.ws_rows + w.tail_row0 + i) * 16;
-#pragma unroll 4
-                for (int c4 = 0; c4 < 16; ++c4) {
-                    p.ws_k[drow + c4] = __ldg(p.k_new + srow + c4);
-                    p.ws_v[drow + c4] = __ldg(p.v_new + srow + c4);
-                }
-            }
-        }
         auto produce = [&](int s, int rope, uint32_t &nEp) {
             const int buf = nEp & 1;
             if (nEp >= 2) {                                 // the epoch before last used this buffer
@@ -709,6 +697,26 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
                 if (k == 0 || rope != prev1) produce(1, rope, nEp1);
                 prev1 = rope;
             }
+        }
+    }
+}
+
+// ---- append (the two spare warps) -------------------------------------------------------------------------------
+// With tail_direct the attention reads the query block's K/V from the caller's tensors; the piece that starts
+// a (request, kv head) also copies those rows behind the prefix in the workspace, for later calls.  Nothing
+// in this launch waits for the copy.
+__device__ __forceinline__ void append_role(const Params &p, const Cta &c, const int t)
+{
+    if (!p.tail_direct) return;
+    for (int wi = c.item_begin; wi < c.item_end; ++wi) {
+        const Work w = load_work(p, wi);
+        if (w.lo != 0 || w.row_base != 0) continue;
+        for (int i = t; i < p.q_len * 16; i += 64) {            // 16-byte words of the rows of this kv head
+            const int row = i >> 4, c4 = i & 15;
+            const long long src = (((long long)w.b * p.q_len + row) * p.n_kv + w.hk) * 16 + c4;
+            const long long dst = ((long long)w.plane * p.ws_rows + w.tail_row0 + row) * 16 + c4;
+            p.ws_k[dst] = __ldg(p.k_new + src);
+            p.ws_v[dst] = __ldg(p.v_new + src);
         }
     }
 }
@@ -1053,6 +1061,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
             mma_role(p, c);
         } else if (warp == 13) {
             tma_role(p, c, lane, &tm_pool_k, &tm_pool_v, &tm_ws_k, &tm_ws_v, &tm_knew, &tm_vnew);
+        } else {
+            append_role(p, c, tid - 448);
         }
     }
 
