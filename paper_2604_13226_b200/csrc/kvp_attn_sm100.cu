@@ -342,58 +342,74 @@ __device__ __forceinline__ int load_seq(int mode, int n, int r, int kv)
     return r <= n - 2 ? 2 * r + 2 : 2 * n - 1;
 }
 
-// Write this thread's query row (128 bf16 = 16 x 16 bytes), counter-rotated by the offset of rope-table
-// row `rope` - q' = R(-Delta) q, which leaves q'.k = q.(R(Delta) k), Eq. 1 moved onto Q - into a rotated-Q
-// buffer in the K-major 128-byte-swizzled layout (two 64-column halves of 128 rows x 128 bytes).
-__device__ __forceinline__ void produce_q_row(const Params &p, char *qbuf, int t, const __nv_bfloat16 *qrow, int rope)
+// The Q producer (128 threads) writes one 128-row query tile, counter-rotated by the offset of rope-table row
+// `rope` - q' = R(-Delta) q, which leaves q'.k = q.(R(Delta) k), Eq. 1 moved onto Q - into a rotated-Q buffer
+// in the K-major 128-byte-swizzled layout (two 64-column halves of 128 rows x 128 bytes).  Thread t owns
+// the 16-byte chunks c = t & 7 and c + 8 (the rotation partners when pairs are (i, i + 64)) of rows
+// t >> 3, + 16, + 32, ...  The raw rows go to their place in the buffer by asynchronous copies, all in flight
+// together (one memory round trip for the tile, eight threads per 128-byte line); the thread then rotates
+// its own chunks in place.
+__device__ __forceinline__ void produce_q_tile(const Params &p, char *qbuf, int t, const __nv_bfloat16 *q_b, int hk,
+                                               int row_base, int n_rows, int rope)
 {
-    const int sw = t & 7;
-    char *row_lo = qbuf + t * 128;
-    char *row_hi = row_lo + kHalfBytes;
-    if (qrow == nullptr) {
+    const int c = t & 7, r0 = t >> 3;
+    char *mine = qbuf + r0 * 128 + ((c ^ (r0 & 7)) << 4);                       // row & 7 == r0 & 7 for all of its rows
+    float4 w4[4];
+    if (rope != 0) {
+        const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
-        }
-        return;
+        for (int j = 0; j < 4; ++j)
+            w4[j] = __ldg(p.pairing == 0 ? cs + c * 4 + j : cs + (c + 8 * (j >> 1)) * 2 + (j & 1));
     }
-    const uint4 *src = reinterpret_cast<const uint4 *>(qrow);
-    const float4 *cs = reinterpret_cast<const float4 *>(p.plan.rope + (size_t)rope * 64);   // (cos, sin) pairs
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i) {
+        const int r = row_base + r0 + 16 * i;
+        char *lo = mine + i * (16 * 128);
+        if (r < n_rows) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(q_b + ((long long)(r / p.group) * p.n_q + hk * p.group + r % p.group) * 128);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(lo)), "l"(src + c) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(lo + kHalfBytes)), "l"(src + c + 8) : "memory");
+        } else {
+            *reinterpret_cast<uint4 *>(lo) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(lo + kHalfBytes) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (rope == 0) return;
     auto lo_f = [](uint32_t u) { return __uint_as_float(u << 16); };
     auto hi_f = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
-        uint4 qa = __ldg(src + c), qb = __ldg(src + c + 8);
+    for (int i = 0; i < 8; ++i) {
+        if (row_base + r0 + 16 * i >= n_rows) break;
+        char *lo = mine + i * (16 * 128);
+        uint4 qa = *reinterpret_cast<uint4 *>(lo), qb = *reinterpret_cast<uint4 *>(lo + kHalfBytes);
         uint32_t *a = reinterpret_cast<uint32_t *>(&qa);
         uint32_t *b = reinterpret_cast<uint32_t *>(&qb);
-        if (rope != 0) {
-            if (p.pairing == 0) {
-                // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
+        if (p.pairing == 0) {
+            // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float4 w = __ldg(cs + c * 4 + j);              // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
-                    const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
-                    a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
-                    b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
-                }
-            } else {
-                // pairs (2i, 2i+1): one word each; chunk c holds pairs 4c..4c+3
+            for (int j = 0; j < 4; ++j) {
+                const float4 w = w4[j];                          // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
+                const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
+                a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
+                b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
+            }
+        } else {
+            // pairs (2i, 2i+1): one word each; chunk c holds pairs 4c..4c+3 (w4[0], w4[1]), chunk c+8 w4[2], w4[3]
 #pragma unroll
-                for (int j = 0; j < 4; j += 2) {
-                    float4 w = __ldg(cs + c * 2 + (j >> 1));
-                    float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
-                    a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
-                    a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
-                    w = __ldg(cs + (c + 8) * 2 + (j >> 1));
-                    x0 = lo_f(b[j]); y0 = hi_f(b[j]); x1 = lo_f(b[j + 1]); y1 = hi_f(b[j + 1]);
-                    b[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
-                    b[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
-                }
+            for (int j = 0; j < 4; j += 2) {
+                float4 w = w4[j >> 1];
+                float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
+                a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+                w = w4[2 + (j >> 1)];
+                x0 = lo_f(b[j]); y0 = hi_f(b[j]); x1 = lo_f(b[j + 1]); y1 = hi_f(b[j + 1]);
+                b[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                b[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
             }
         }
-        *reinterpret_cast<uint4 *>(row_lo + ((c ^ sw) << 4)) = qa;
-        *reinterpret_cast<uint4 *>(row_hi + ((c ^ sw) << 4)) = qb;
+        *reinterpret_cast<uint4 *>(lo) = qa;
+        *reinterpret_cast<uint4 *>(lo + kHalfBytes) = qb;
     }
 }
 
@@ -677,11 +693,8 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
             }
-            const int r = w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0) + t;
-            const __nv_bfloat16 *qrow = nullptr;
-            if (r < n_rows)
-                qrow = p.q + (((long long)w.b * p.q_len + r / p.group) * p.n_q + w.hk * p.group + r % p.group) * 128;
-            produce_q_row(p, c.smem + kOffQ + (2 * s + buf) * kTileBytes, t, qrow, rope);
+            produce_q_tile(p, c.smem + kOffQ + (2 * s + buf) * kTileBytes, t, p.q + (long long)w.b * p.q_len * p.n_q * 128,
+                           w.hk, w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0), n_rows, rope);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(c.bar(kQFull + 2 * s + buf));
             ++nEp;
