@@ -24,6 +24,7 @@
 //                     then S = Q K^T of the next one; the two streams alternate.
 //   warp 13           TMA producer: K and V tiles into a 3-stage ring (two 64-column boxes each,
 //                     128-byte swizzle), in the order the MMA warp consumes them.
+//   warps 14-15       with tail_direct: copy the query block's K/V rows behind the prefix (the append).
 //
 // Every mbarrier wait is bounded: when it runs out the CTA records a code in the status word, drains
 // what it has in flight, frees TMEM and returns.
