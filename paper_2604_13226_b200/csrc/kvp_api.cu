@@ -245,15 +245,15 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     // budget that needs no more than G CTAs is found by bisection.
     struct cut_t { int32_t u, t; };
     std::vector<cut_t> cuts;
-    auto fill = [&](int64_t budget, std::vector<cut_t> *rec) -> int {
+    auto fill = [&](size_t u_begin, size_t u_end, int64_t budget, std::vector<cut_t> *rec) -> int {
         int used = 0;
-        size_t u = 0;
+        size_t u = u_begin;
         int32_t t = 0;
-        while (u < units.size()) {
+        while (u < u_end) {
             ++used;
             if (rec) rec->push_back({(int32_t)u, t});
             int64_t cost = 0;
-            while (u < units.size()) {
+            while (u < u_end) {
                 const int w = units[u].mode ? 1 : 2;
                 const int32_t left = units[u].n_all - t;
                 const int64_t room = budget - cost - kPieceCost;
@@ -274,12 +274,48 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
         }
         return used;
     };
-    int64_t lo_b = std::max<int64_t>(total / G, 8 + kPieceCost), hi_b = total + kPieceCost;
-    while (lo_b < hi_b) {
-        const int64_t mid = (lo_b + hi_b) / 2;
-        if (fill(mid, nullptr) <= G) hi_b = mid; else lo_b = mid + 1;
+    auto cut_range = [&](size_t u_begin, size_t u_end, int64_t weight, int g) {
+        int64_t lo_b = std::max<int64_t>(weight / g, 8 + kPieceCost), hi_b = weight + kPieceCost;
+        while (lo_b < hi_b) {
+            const int64_t mid = (lo_b + hi_b) / 2;
+            if (fill(u_begin, u_end, mid, nullptr) <= g) hi_b = mid; else lo_b = mid + 1;
+        }
+        fill(u_begin, u_end, lo_b, &cuts);
+    };
+    // Each row block gets its own run of CTAs, in proportion to its work, and is cut on its own: row blocks of
+    // equal work then get the same cuts, so the CTAs of units that share K/V walk the same tiles in step.  With
+    // more row blocks than half the CTAs (or when told not to split) the whole line is cut at once.
+    std::vector<size_t> rb_begin;                                 // first unit of every row block
+    std::vector<int64_t> rb_weight;
+    for (size_t u = 0; u < units.size(); ++u) {
+        if (u == 0 || units[u].row_base != units[u - 1].row_base) {
+            rb_begin.push_back(u);
+            rb_weight.push_back(0);
+        }
+        rb_weight.back() += (int64_t)units[u].n_all * (units[u].mode ? 1 : 2) + kPieceCost;
     }
-    fill(lo_b, &cuts);
+    rb_begin.push_back(units.size());
+    const int n_rb = (int)rb_weight.size();
+    std::vector<int> rb_ctas(n_rb, 0);
+    bool per_block = n_rb >= 2 && 2 * n_rb <= G && !no_split;
+    if (per_block) {
+        int given = 0;
+        std::vector<std::pair<int64_t, int>> rem;
+        for (int r = 0; r < n_rb; ++r) {
+            const int64_t num = rb_weight[r] * G;
+            rb_ctas[r] = (int)(num / total);
+            rem.push_back({-(num % total), r});
+            given += rb_ctas[r];
+        }
+        std::sort(rem.begin(), rem.end());
+        for (int i = 0; given < G; ++i, ++given) ++rb_ctas[rem[i % n_rb].second];
+        for (int r = 0; r < n_rb; ++r) per_block = per_block && rb_ctas[r] >= 1;
+    }
+    if (per_block) {
+        for (int r = 0; r < n_rb; ++r) cut_range(rb_begin[r], rb_begin[r + 1], rb_weight[r], rb_ctas[r]);
+    } else {
+        cut_range(0, units.size(), total, G);
+    }
     cuts.push_back({(int32_t)units.size(), 0});
 
     std::vector<kvp_work> &works = out.works;
