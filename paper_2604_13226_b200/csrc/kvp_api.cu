@@ -311,8 +311,13 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
         for (int i = 0; given < G; ++i, ++given) ++rb_ctas[rem[i % n_rb].second];
         for (int r = 0; r < n_rb; ++r) per_block = per_block && rb_ctas[r] >= 1;
     }
+    std::vector<int> rb_used(n_rb, 0);
     if (per_block) {
-        for (int r = 0; r < n_rb; ++r) cut_range(rb_begin[r], rb_begin[r + 1], rb_weight[r], rb_ctas[r]);
+        for (int r = 0; r < n_rb; ++r) {
+            const size_t before = cuts.size();
+            cut_range(rb_begin[r], rb_begin[r + 1], rb_weight[r], rb_ctas[r]);
+            rb_used[r] = (int)(cuts.size() - before);
+        }
     } else {
         cut_range(0, units.size(), total, G);
     }
@@ -320,9 +325,11 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
 
     std::vector<kvp_work> &works = out.works;
     std::vector<int32_t> &cta_begin = out.cta_begin;
+    struct cta_rec { std::vector<kvp_work> ws; std::vector<int32_t> unit; };
+    std::vector<cta_rec> recs;
     for (size_t c = 0; c + 1 < cuts.size(); ++c) {
         const cut_t a = cuts[c], z = cuts[c + 1];
-        const size_t before = works.size();
+        cta_rec rec;
         for (int32_t u = a.u; u <= z.u && u < (int32_t)units.size(); ++u) {
             const int32_t lo = (u == a.u) ? a.t : 0;
             const int32_t hi = (u == z.u) ? z.t : units[u].n_all;
@@ -330,23 +337,45 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
             kvp_work w;
             w.b = units[u].b; w.hk = units[u].hk; w.row_base = units[u].row_base; w.mode = units[u].mode;
             w.tile_lo = lo; w.n_tiles = hi - lo; w.slot0 = w.slot1 = -1;
-            if (units[u].n_pieces == 0) units[u].first_piece = (int32_t)works.size();
-            ++units[u].n_pieces;
-            works.push_back(w);
+            rec.ws.push_back(w);
+            rec.unit.push_back(u);
         }
-        if (works.size() > before) cta_begin.push_back((int32_t)before);
+        recs.push_back(rec);
     }
+    // emission order: the j-th CTAs of all row blocks next to each other
+    std::vector<int> order;
+    if (per_block) {
+        std::vector<int> off(n_rb + 1, 0);
+        for (int r = 0; r < n_rb; ++r) off[r + 1] = off[r] + rb_used[r];
+        for (int j = 0; (int)order.size() < off[n_rb]; ++j)
+            for (int r = 0; r < n_rb; ++r)
+                if (j < rb_used[r]) order.push_back(off[r] + j);
+    } else {
+        for (size_t c = 0; c < recs.size(); ++c) order.push_back((int)c);
+    }
+    std::vector<std::vector<int32_t>> unit_pieces(units.size());
+    for (int idx : order) {
+        const cta_rec &rec = recs[idx];
+        if (rec.ws.empty()) continue;
+        cta_begin.push_back((int32_t)works.size());
+        for (size_t i = 0; i < rec.ws.size(); ++i) {
+            unit_pieces[rec.unit[i]].push_back((int32_t)works.size());
+            works.push_back(rec.ws[i]);
+        }
+    }
+    for (size_t u = 0; u < units.size(); ++u) units[u].n_pieces = (int32_t)unit_pieces[u].size();
     const int n_ctas = (int)cta_begin.size();
     cta_begin.push_back((int32_t)works.size());
 
     std::vector<kvp_merge_item> &merges = out.merges;
     int32_t n_slots = 0, max_pieces = 1;
-    for (const unit_t &u : units) {
+    for (size_t ui = 0; ui < units.size(); ++ui) {
+        const unit_t &u = units[ui];
         if (u.n_pieces <= 1) continue;
         max_pieces = std::max(max_pieces, u.n_pieces);
         const int32_t base = n_slots;
         for (int i = 0; i < u.n_pieces; ++i) {
-            kvp_work &w = works[u.first_piece + i];      // the pieces of a unit are consecutive
+            kvp_work &w = works[unit_pieces[ui][i]];
             w.slot0 = base + i;
             if (u.mode == 0) w.slot1 = base + u.n_pieces + i;
         }

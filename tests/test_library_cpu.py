@@ -227,28 +227,24 @@ def test_compressed_registration_and_per_layer_lists_host_only():
     assert e.value.code == 4
 
 
-def test_schedule_puts_units_that_share_keys_a_whole_number_of_ctas_apart():
-    # Config-3 shape: every (request, kv head) has two 256-row units that stream the same K/V.  Row blocks are the
-    # outermost order of the work list and two divides the CTA count, so the second unit's pieces repeat the first
-    # one's cuts 74 CTAs further on: the two CTAs reach the same key tiles at the same time.
+def test_schedule_gives_units_that_share_keys_the_same_cuts_on_neighbouring_ctas():
+    # Config-3 shape: every (request, kv head) has two 256-row units that stream the same K/V.  Each row block is
+    # cut on its own run of CTAs, so the second unit's pieces repeat the first one's cuts, and the j-th CTAs of the
+    # row blocks are emitted next to each other: the two CTAs reach the same key tiles at the same time.
     ctx, aid, plen, shape = _schedule_case(32, 8, [1024] * 10, [[(i, 0) for i in range(10)]] * 4, 128)
     cb, works, merges, n_slots = ctx.export_schedule(aid, 128)
     n_ctas = len(cb) - 1
     assert n_ctas == 148
-    row_bases = [int(w[2]) for w in works]
-    assert row_bases == sorted(row_bases)                       # all row-block-0 pieces come first
-    first = {}
+    pieces = {}
     for c in range(n_ctas):
         for i in range(cb[c], cb[c + 1]):
             b, hk, row_base, mode, lo, n = (int(x) for x in works[i][:6])
-            first.setdefault((b, hk, row_base), []).append((c, lo, n))
-    near = 0
-    for (b, hk, row_base), pieces in first.items():
+            pieces.setdefault((b, hk, row_base), []).append((c, lo, n))
+    for (b, hk, row_base), first in pieces.items():
         if row_base != 0:
             continue
-        for (c0, lo0, n0), (c1, lo1, n1) in zip(pieces, first[(b, hk, 256)]):
-            assert c1 - c0 in (73, 74, 75)
-            near += abs(lo1 - lo0) <= 2
-    assert near >= 0.9 * sum(len(v) for k, v in first.items() if k[2] == 0)
+        second = pieces[(b, hk, 256)]
+        assert len(first) == len(second)
+        for (c0, lo0, n0), (c1, lo1, n1) in zip(first, second):
+            assert (c1, lo1, n1) == (c0 + 1, lo0, n0)
     ctx.close()
-
