@@ -298,6 +298,62 @@ def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: fl
             "l2": "flushed between iterations"}
 
 
+def measure_host_packets_point(seed: int, iters: int, device: int, n_layers: int = 8):
+    """Config-3 shape with `n_layers` layers and every packet waiting in pinned host memory: one request batch from
+    `kvp_assemble` (which starts the host-to-pool copies, layer by layer) to the last layer's attention, against the
+    same step with the packets resident and against the bare copy time.  The attention of layer l overlaps the copy
+    of the layers after it; the link decides the total."""
+    import torch
+    from paper_2604_13226_b200 import inputs as gen
+    from paper_2604_13226_b200.session import Session
+    spec = gen.spec_config3(seed=seed, n_layers=n_layers)
+    wl = gen.DeviceWorkload(spec, f"cuda:{device}")
+    dev = torch.device(f"cuda:{device}")
+    sess = Session(wl, device=device, host_packets=True)
+    qkv = [sess.query_tensors(l) for l in range(n_layers)]
+    n_packets = len(spec.packet_lens)
+    used = sorted({pid for item in wl.items for pid, _ in item})          # only the packets a request names are copied
+    h2d = sum(sess.host_kv[pid][0].numel() * sess.host_kv[pid][0].element_size() * 2 for pid in used)
+
+    def step(evict):
+        if evict:
+            for pid in range(n_packets):
+                sess.ctx.evict_packet(pid)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sess.assemble()
+        for l in range(n_layers):
+            sess.prefill(l, qkv=qkv[l], want_lse=False)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1)
+
+    step(True)
+    cold = statistics.median(step(True) for _ in range(iters))
+    warm = statistics.median(step(False) for _ in range(iters))
+    # the bare transfer: the same pinned buffers to a device buffer of the same size
+    sink = [(torch.empty_like(hk, device=dev), torch.empty_like(hv, device=dev)) for hk, hv in sess.host_kv[:4]]
+    torch.cuda.synchronize(dev)
+    ts = []
+    for _ in range(iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for (dk, dv), (hk, hv) in zip(sink, sess.host_kv[:4]):
+            dk.copy_(hk, non_blocking=True)
+            dv.copy_(hv, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ts.append(e0.elapsed_time(e1))
+    link_gbs = sum(hk.numel() * hk.element_size() * 2 for hk, _ in sess.host_kv[:4]) / statistics.median(ts) / 1e6
+    assert sess.ctx.status_word() == 0
+    sess.close()
+    del sess, wl, sink
+    torch.cuda.empty_cache()
+    return {"workload": f"config3 shape, {n_layers} layers, packets in pinned host memory", "h2d_bytes": h2d,
+            "assemble_to_last_layer_ms": cold, "h2d_gbs_inside_it": h2d / cold / 1e6, "plain_copy_gbs": link_gbs,
+            "same_step_packets_resident_ms": warm}
+
+
 # ---------------------------------------------------------------------------------------------------
 # main
 # ---------------------------------------------------------------------------------------------------
@@ -542,6 +598,7 @@ def main():
                 # the step after the prefill: one new token per request over 16 x 33,280-token composed caches
                 extras["decode_point"] = measure_point("config5:16:1:16", args.seed, 10, False, peaks, local_rank)
                 extras["compressed_point"] = measure_compressed_point(args.seed, 10, peaks, local_rank)
+                extras["host_packets_point"] = measure_host_packets_point(args.seed, 5, local_rank)
             except Exception as ex:                                   # extras never invalidate the main line
                 extras["error"] = repr(ex)
             line["extra_points"] = extras

@@ -119,6 +119,30 @@ KVP_API int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, 
                             int32_t cache_pos0, void *stream, int32_t *packet_id);
 
 /*
+ * Register one packet whose K/V stay in host memory until a request uses it (the CPU-to-GPU cache transfer
+ * that the paper counts inside time-to-first-token, Section 4.3).  Pool rows are reserved now; nothing is copied.
+ * The first kvp_assemble that names the packet enqueues the copy on a stream the context owns, layer by layer,
+ * and kvp_query_prefill(layer) makes its stream wait for that layer only: the transfer of layer l+1 runs while
+ * layer l is attended to.  After that the packet is resident like any other, until kvp_evict_packet.
+ *   k_host, v_host   host, layout [n_layers][n_kv_heads][n_tokens][head_dim] (the pool's own plane order, so a
+ *                    layer of a packet is one strided copy); k post-RoPE for positions cache_pos0 + t.  The
+ *                    buffers stay with the caller and must remain valid while the packet is registered; pinned
+ *                    memory is needed for the copies to overlap anything.
+ * In a host-only context the pointers may be NULL.  Not available for compressed packets.
+ * Errors: INVALID, CAPACITY (max_packets or pool full).
+ */
+KVP_API int32_t kvp_register_packet_host(kvp_ctx *ctx, const void *k_host, const void *v_host, int32_t n_tokens,
+                                 int32_t cache_pos0, int32_t *packet_id);
+
+/*
+ * Mark a packet registered with kvp_register_packet_host as no longer on the device: the next kvp_assemble
+ * that names it copies it in again (into the same pool rows).  The caller must not evict a packet that work
+ * already enqueued still reads, other than on the stream it passes to that next kvp_assemble.
+ * Errors: NOT_FOUND, STATE (the packet has no host copy).
+ */
+KVP_API int32_t kvp_evict_packet(kvp_ctx *ctx, int32_t packet_id);
+
+/*
  * Register one compressed packet: a document cache after unstructured KV pruning (Section 4.3,
  * "Compatibility with KV Compression": compressors keep a different token subset per layer - and, for
  * many of them, per head - and the method composes such caches as opaque units).  Layer l, kv head h keeps

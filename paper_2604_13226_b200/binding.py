@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         "kvp_destroy": (i32, [vp]),
         "kvp_register_packet": (i32, [vp, vp, vp, i32, i32, vp, pi32]),
         "kvp_register_packet_compressed": (i32, [vp, vp, vp, i32, i32, pi32, vp, pi32]),
+        "kvp_register_packet_host": (i32, [vp, vp, vp, i32, i32, pi32]),
+        "kvp_evict_packet": (i32, [vp, i32]),
         "kvp_register_adapter": (i32, [vp, vp, vp, i32, i32, vp, vp, i32, i32, vp, pi32]),
         "kvp_assemble": (i32, [vp, i32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
         "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
@@ -89,7 +91,8 @@ def lib() -> ctypes.CDLL:
 
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
-            "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
+            "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_packet_host", "kvp_evict_packet",
+            "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
             "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_segment_mass", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
@@ -196,6 +199,17 @@ class Context:
         self._check(self._L.kvp_register_packet_compressed(self._h, _ptr(k), _ptr(v), n_tokens, cache_pos0,
                                                            _i32_array(list(kept)), self._stream(stream), ctypes.byref(out)))
         return out.value
+
+    def register_packet_host(self, k_host, v_host, n_tokens: int, cache_pos0: int = 0) -> int:
+        """k_host, v_host: host tensors [n_layers][n_kv_heads][n_tokens][head_dim] (pinned for overlap), kept alive
+        by the caller; they are copied into the pool by the first assemble that names the packet."""
+        out = ctypes.c_int32(-1)
+        self._check(self._L.kvp_register_packet_host(self._h, _ptr(k_host), _ptr(v_host), n_tokens, cache_pos0,
+                                                     ctypes.byref(out)))
+        return out.value
+
+    def evict_packet(self, packet_id: int) -> None:
+        self._check(self._L.kvp_evict_packet(self._h, packet_id))
 
     def register_adapter(self, hk, hv, n_header: int, header_pos0: int, tk, tv, n_trailer: int,
                          trailer_pos0: int, stream=None) -> int:

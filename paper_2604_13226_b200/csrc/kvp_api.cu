@@ -555,6 +555,14 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
         ctx->sched_event.push_back(evs);
     }
 
+    if (cudaStreamCreateWithFlags(&ctx->load_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->load_fence, cudaEventDisableTiming) != cudaSuccess)
+        return bail(KVP_ERR_CUDA, "load stream creation failed");
+    ctx->load_done.resize(sh.n_layers);
+    for (int l = 0; l < sh.n_layers; ++l)
+        if (cudaEventCreateWithFlags(&ctx->load_done[l], cudaEventDisableTiming) != cudaSuccess)
+            return bail(KVP_ERR_CUDA, "load event creation failed");
+
     if (sh.dtype == KVP_DTYPE_BF16 && sh.head_dim == 128 && prop.major == 10) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -590,6 +598,9 @@ int32_t kvp_destroy(kvp_ctx *ctx)
         for (char *h : ctx->slot_sched_host) cudaFreeHost(h);
         for (cudaEvent_t e : ctx->sched_event) cudaEventDestroy(e);
         for (auto &w : ctx->tev) for (auto &v : w) for (cudaEvent_t e : v) cudaEventDestroy(e);
+        for (cudaEvent_t e : ctx->load_done) cudaEventDestroy(e);
+        if (ctx->load_fence) cudaEventDestroy(ctx->load_fence);
+        if (ctx->load_stream) cudaStreamDestroy(ctx->load_stream);
     }
     delete ctx;
     return KVP_OK;
@@ -617,6 +628,66 @@ int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t 
     ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0, {}});
     ctx->pool_rows_used += n_tokens;
     *packet_id = (int32_t)ctx->packets.size() - 1;
+    return KVP_OK;
+}
+
+int32_t kvp_register_packet_host(kvp_ctx *ctx, const void *k_host, const void *v_host, int32_t n_tokens,
+                                 int32_t cache_pos0, int32_t *packet_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!packet_id || n_tokens <= 0) return fail(ctx, KVP_ERR_INVALID, "register_packet_host: bad arguments");
+    if (!ctx->host_only && (!k_host || !v_host)) return fail(ctx, KVP_ERR_INVALID, "register_packet_host: null K/V");
+    if ((int)ctx->packets.size() >= ctx->cfg.max_packets) return fail(ctx, KVP_ERR_CAPACITY, "max_packets reached");
+    if (ctx->pool_rows_used + n_tokens > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
+    ctx->packets.push_back({(int32_t)ctx->pool_rows_used, n_tokens, cache_pos0, {}});
+    ctx->pool_rows_used += n_tokens;
+    ctx->packet_src.resize(ctx->packets.size());
+    kvp_ctx::host_src &src = ctx->packet_src.back();
+    src.k = (const char *)k_host;
+    src.v = (const char *)v_host;
+    src.from_host = true;
+    src.resident = false;
+    *packet_id = (int32_t)ctx->packets.size() - 1;
+    return KVP_OK;
+}
+
+int32_t kvp_evict_packet(kvp_ctx *ctx, int32_t packet_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (packet_id < 0 || packet_id >= (int)ctx->packets.size()) return fail(ctx, KVP_ERR_NOT_FOUND, "evict_packet: unknown packet id %d", packet_id);
+    if (packet_id >= (int)ctx->packet_src.size() || !ctx->packet_src[packet_id].from_host)
+        return fail(ctx, KVP_ERR_STATE, "evict_packet: packet %d has no host copy to come back from", packet_id);
+    ctx->packet_src[packet_id].resident = false;
+    return KVP_OK;
+}
+
+// Host -> pool copies of the packets of an assembly that are not on the device yet, one layer after the other
+// on the context's own stream, an event per layer.  Host layout [n_layers][n_kv_heads][n_tokens][head_dim]: a
+// layer of a packet is n_kv_heads runs of n_tokens rows, one per plane, i.e. one 2-D copy for K and one for V.
+static int32_t load_host_packets(kvp_ctx *ctx, const std::vector<int32_t> &ids, cudaStream_t st)
+{
+    const kvp_shape &sh = ctx->shape;
+    const size_t row_bytes = (size_t)sh.head_dim * sh.elem_bytes;
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    // the rows may still be read by work the caller enqueued before (a packet that was evicted)
+    KVP_CUDA(ctx, cudaEventRecord(ctx->load_fence, st));
+    KVP_CUDA(ctx, cudaStreamWaitEvent(ctx->load_stream, ctx->load_fence, 0));
+    for (int l = 0; l < sh.n_layers; ++l) {
+        for (int32_t id : ids) {
+            const kvp_segment_host &pk = ctx->packets[id];
+            const kvp_ctx::host_src &src = ctx->packet_src[id];
+            const size_t run = (size_t)pk.n * row_bytes;
+            const size_t dst = ((size_t)l * sh.n_kv_heads * sh.pool_rows + pk.row0) * row_bytes;
+            const size_t from = (size_t)l * sh.n_kv_heads * run;
+            KVP_CUDA(ctx, cudaMemcpy2DAsync(ctx->pool_k + dst, (size_t)sh.pool_rows * row_bytes, src.k + from, run, run,
+                                            sh.n_kv_heads, cudaMemcpyHostToDevice, ctx->load_stream));
+            KVP_CUDA(ctx, cudaMemcpy2DAsync(ctx->pool_v + dst, (size_t)sh.pool_rows * row_bytes, src.v + from, run, run,
+                                            sh.n_kv_heads, cudaMemcpyHostToDevice, ctx->load_stream));
+        }
+        KVP_CUDA(ctx, cudaEventRecord(ctx->load_done[l], ctx->load_stream));
+    }
+    for (int32_t id : ids) ctx->packet_src[id].resident = true;
+    ctx->loads_recorded = true;
     return KVP_OK;
 }
 
@@ -705,6 +776,17 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
     kvp_assembly_host as;
     as.flags = flags;
     as.batch = batch;
+    // packets that still wait in host memory are brought in now, layer by layer, on the context's own stream
+    std::vector<int32_t> to_load;
+    bool host_origin = false;
+    for (int s = 0; s < n_slots; ++s) {
+        const int32_t id = packet_ids[s];
+        if (id >= (int)ctx->packet_src.size() || !ctx->packet_src[id].from_host) continue;
+        host_origin = true;
+        if (!ctx->packet_src[id].resident && std::find(to_load.begin(), to_load.end(), id) == to_load.end()) to_load.push_back(id);
+    }
+    as.waits_loads = host_origin && !ctx->host_only && (ctx->loads_recorded || !to_load.empty());
+    const bool waits_loads = as.waits_loads;
     std::map<int32_t, int32_t> rope_of;        // delta -> rope-table index (0 = identity)
     std::vector<int32_t> rope_delta(1, 0);
     rope_of[0] = 0;
@@ -872,8 +954,16 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
     const int32_t n_chunks = as.n_chunks;
     ctx->slots[slot] = std::move(as);
     *assembly_id = id;
-    if (!ctx->host_only) {
+    if (ctx->host_only) {
+        for (int32_t id : to_load) ctx->packet_src[id].resident = true;
+    } else {
         cudaStream_t st = (cudaStream_t)stream;
+        if (!to_load.empty()) {
+            const int32_t rc = load_host_packets(ctx, to_load, st);
+            if (rc != KVP_OK) return rc;
+        }
+        if (mat && waits_loads)                                   // the gather reads every layer of the documents
+            KVP_CUDA(ctx, cudaStreamWaitEvent(st, ctx->load_done[ctx->shape.n_layers - 1], 0));
         KVP_CUDA(ctx, time_edge(ctx, 1, 0, st));
         KVP_CUDA(ctx, kvp_launch_gather(ctx->shape, plan_dev(ctx, slot), n_chunks, ctx->pool_k, ctx->pool_v,
                                         ctx->slot_k[slot], ctx->slot_v[slot], st));
@@ -919,6 +1009,7 @@ int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32
         n_query_rows > ctx->cfg.max_query_tokens)
         return fail(ctx, KVP_ERR_INVALID, "export_cache: bad arguments");
     KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (as.waits_loads) KVP_CUDA(ctx, cudaStreamWaitEvent((cudaStream_t)stream, ctx->load_done[layer], 0));
     KVP_CUDA(ctx, kvp_launch_export(ctx->shape, plan_dev(ctx, slot), b, layer, as.items[b].prefix_len, n_query_rows,
                                     ctx->pool_k, ctx->pool_v, ctx->slot_k[slot], ctx->slot_v[slot], k_out, v_out,
                                     k_as_f32, (cudaStream_t)stream));
@@ -944,6 +1035,7 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     if (q_pos0 + q_len > ctx->cfg.max_query_tokens)
         return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: %d rows appended + q_len %d > max_query_tokens", q_pos0, q_len);
     KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (as.waits_loads) KVP_CUDA(ctx, cudaStreamWaitEvent(st, ctx->load_done[layer], 0));   // this layer's documents have landed
     const kvp_plan_dev plan = plan_dev(ctx, slot);
     const int rope_query = (flags & KVP_ROPE_QUERY) ? 1 : 0;
     const double *inv_freq_dev = reinterpret_cast<const double *>((char *)ctx->cfg.workspace + 256);
@@ -1078,6 +1170,7 @@ int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const
     for (int b = 0; b < as.batch; ++b) max_seg = std::max(max_seg, as.items[b].seg_end - as.items[b].seg_begin);
     if (n_cols <= max_seg) return fail(ctx, KVP_ERR_CAPACITY, "segment_mass: n_cols %d <= %d segments", n_cols, max_seg);
     KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (as.waits_loads) KVP_CUDA(ctx, cudaStreamWaitEvent((cudaStream_t)stream, ctx->load_done[layer], 0));
     const void *q_used = (flags & KVP_ROPE_QUERY) ? (const void *)ctx->q_scratch : q;
     KVP_CUDA(ctx, kvp_launch_segment_mass(ctx->shape, plan_dev(ctx, slot), as.batch, q_len, as.appended[layer] - q_len, layer,
                                           q_used, lse, ctx->pool_k, ctx->slot_k[slot], mass, n_cols, (cudaStream_t)stream));

@@ -117,6 +117,7 @@ struct kvp_assembly_host {
     int32_t item_stride = 0;               // batch when the assembly has per-layer tile lists (compressed packets)
     int32_t last_q_len = 0;
     std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
+    bool waits_loads = false;              // uses packets that came from host memory: wait for the layer's load event
     // work lists of the two-stream kernel (one, or one per layer when the tile lists differ per layer), each
     // built for q_len query tokens at offset q_pos0 (q_len 0 = none yet)
     struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; };
@@ -129,6 +130,13 @@ struct kvp_ctx {
     bool host_only = false;
     std::vector<double> inv_freq;
     std::vector<kvp_segment_host> packets;
+    // packets whose K/V wait in host memory until a request uses them (parallel to `packets`, grown on demand)
+    struct host_src { const char *k = nullptr, *v = nullptr; bool from_host = false, resident = true; };
+    std::vector<host_src> packet_src;
+    cudaStream_t load_stream = nullptr;             // host -> pool copies, layer by layer
+    cudaEvent_t load_fence = nullptr;               // the caller's stream at the assemble that starts a load
+    std::vector<cudaEvent_t> load_done;             // [layer]: the loads enqueued so far have landed for this layer
+    bool loads_recorded = false;
     std::vector<kvp_segment_host> adapter_h, adapter_t;
     int64_t pool_rows_used = 0;
 

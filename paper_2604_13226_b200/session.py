@@ -32,7 +32,7 @@ def torch_to_np(t, dtype: str) -> np.ndarray:
 
 class Session:
     def __init__(self, wl, materialize: bool = False, device: int = 0, max_query_tokens: Optional[int] = None,
-                 max_assemblies: int = 1):
+                 max_assemblies: int = 1, host_packets: bool = False):
         import torch
         self.torch = torch
         self.wl = wl
@@ -65,10 +65,18 @@ class Session:
                                max_ws_rows=ws_rows + 8, max_assemblies=max_assemblies, device=device,
                                max_compressed=0 if is_dev else sum(1 for p in wl.packets if p.kept is not None))
         # registration (offline in the paper; not part of any timed region)
+        self.host_kv = []                      # pinned host copies of the packets (host_packets): kept alive here
         if is_dev:
             for pid in range(len(lens)):
                 k, v = wl.packet_device(pid)
-                self.ctx.register_packet(k, v, lens[pid], 0)
+                if host_packets:
+                    # [layers][tokens][kv heads][d] -> the pool's plane order [layers][kv heads][tokens][d], in pinned memory
+                    hk = k.permute(0, 2, 1, 3).contiguous().cpu().pin_memory()
+                    hv = v.permute(0, 2, 1, 3).contiguous().cpu().pin_memory()
+                    self.host_kv.append((hk, hv))
+                    self.ctx.register_packet_host(hk, hv, lens[pid], 0)
+                else:
+                    self.ctx.register_packet(k, v, lens[pid], 0)
                 del k, v
             hk, hv, tk, tv = wl.adapter_device()
             self.ctx.register_adapter(hk, hv, wl.spec.n_header, 0, tk, tv, wl.spec.n_trailer, 0)
@@ -82,6 +90,12 @@ class Session:
                     k = np_to_torch(np.concatenate(runs_k, axis=0), s.dtype, self.device)
                     v = np_to_torch(np.concatenate(runs_v, axis=0), s.dtype, self.device)
                     self.ctx.register_packet_compressed(k, v, p.n_tokens, p.cache_pos0, counts)
+                    continue
+                if host_packets:
+                    hk = np_to_torch(np.ascontiguousarray(np.transpose(p.k, (0, 2, 1, 3))), s.dtype, "cpu").pin_memory()
+                    hv = np_to_torch(np.ascontiguousarray(np.transpose(p.v, (0, 2, 1, 3))), s.dtype, "cpu").pin_memory()
+                    self.host_kv.append((hk, hv))
+                    self.ctx.register_packet_host(hk, hv, p.n_tokens, p.cache_pos0)
                     continue
                 k = np_to_torch(p.k, s.dtype, self.device)
                 v = np_to_torch(p.v, s.dtype, self.device)

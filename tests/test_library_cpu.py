@@ -248,3 +248,30 @@ def test_schedule_gives_units_that_share_keys_the_same_cuts_on_neighbouring_ctas
         for (c0, lo0, n0), (c1, lo1, n1) in zip(first, second):
             assert (c1, lo1, n1) == (c0 + 1, lo0, n0)
     ctx.close()
+
+
+def test_packets_registered_from_host_memory_plan_like_any_other():
+    # host-only context: nothing is copied, but rows are reserved in the same order and the plan is the same;
+    # only packets that came from host memory can be evicted
+    shape = gen.ModelShape(2, 8, 2, 128, "bf16", 500000.0)
+    wl = gen.make_workload(shape, [200, 37, 300], [[(0, 0), (2, 0)], [(1, 0), (0, -1)]], q_len=8, n_header=16, n_trailer=16, seed=2)
+    a = host_ctx(shape, wl)
+    aid_a, plen_a = a.assemble(wl.items, kvp.REBASE)
+    b = kvp.Context(shape.n_layers, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.dtype, rope_theta=shape.rope_theta,
+                    pool_tokens=1000, max_packets=3, max_adapters=1, max_batch=2, max_slots=4, max_prefix_tokens=1000,
+                    max_query_tokens=8, max_ws_rows=1200, device=-1)
+    for p_ in wl.packets:
+        b.register_packet_host(None, None, p_.n_tokens, p_.cache_pos0)
+    ad = wl.adapters[0]
+    b.register_adapter(None, None, ad.n_header, ad.header_pos0, None, None, ad.n_trailer, ad.trailer_pos0)
+    aid_b, plen_b = b.assemble(wl.items, kvp.REBASE)
+    assert plen_a == plen_b
+    for i in range(2):
+        pa, pb = a.export_plan(aid_a, i), b.export_plan(aid_b, i)
+        assert all(np.array_equal(x, y) for x, y in zip(pa, pb))
+    b.evict_packet(1)
+    with pytest.raises(kvp.KvpError):
+        a.evict_packet(1)
+    a.close()
+    b.close()
+
