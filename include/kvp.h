@@ -286,8 +286,9 @@ KVP_API int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int3
    key KVP_TUNE_FUSED_APPEND: 1 (default) = on the plain prefill path (no KVP_ROPE_QUERY, no KVP_CONTINUE) the
    tcgen05 kernel reads the query block's keys and values straight from k_new / v_new and appends them itself,
    0 = always run the separate append kernel first;
-   key KVP_TUNE_TIME_KERNELS: value != 0 brackets every attention and gather kernel with CUDA events
-   on the caller's stream (up to 4096 launches between two kvp_kernel_times calls). */
+   key KVP_TUNE_TIME_KERNELS: value p >= 1 brackets every p-th attention kernel and every p-th gather kernel
+   with CUDA events on the caller's stream (up to 4096 timed launches between two kvp_kernel_times calls; the
+   events between back-to-back launches cost a little, hence the period), 0 = off. */
 enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3, KVP_TUNE_KERNEL_VARIANT = 4,
        KVP_TUNE_FUSED_APPEND = 5 };
 KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);

@@ -156,10 +156,13 @@ bool make_query_tensor_map(encode_tiled_fn enc, CUtensorMap *tm, const void *bas
 
 constexpr int kMaxTimed = 4096;
 
-// Record an event before (edge 0) / after (edge 1) a timed kernel; events are created on first use.
+// Record an event before (edge 0) / after (edge 1) a timed kernel; events are created on first use.  With a
+// period p only every p-th kernel of its kind is bracketed.
 cudaError_t time_edge(kvp_ctx *ctx, int which, int edge, cudaStream_t st)
 {
     if (!ctx->time_kernels || ctx->tev_n[which] >= kMaxTimed) return cudaSuccess;
+    if (edge == 0) ctx->tev_open[which] = (ctx->tev_seen[which]++ % ctx->time_kernels) == 0;
+    if (!ctx->tev_open[which]) return cudaSuccess;
     std::vector<cudaEvent_t> &v = ctx->tev[which][edge];
     const int i = ctx->tev_n[which];
     if ((int)v.size() <= i) {
@@ -1249,7 +1252,11 @@ int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
         if (value != 0 && value != 1) return fail(ctx, KVP_ERR_INVALID, "tune: kernel variant %d", value);
         ctx->kernel_variant = value;
     }
-    else if (key == KVP_TUNE_TIME_KERNELS) { ctx->time_kernels = value != 0; ctx->tev_n[0] = ctx->tev_n[1] = 0; }
+    else if (key == KVP_TUNE_TIME_KERNELS) {
+        ctx->time_kernels = std::max(0, value);
+        ctx->tev_n[0] = ctx->tev_n[1] = 0;
+        ctx->tev_seen[0] = ctx->tev_seen[1] = 0;
+    }
     else return fail(ctx, KVP_ERR_INVALID, "tune: unknown key %d", key);
     return KVP_OK;
 }

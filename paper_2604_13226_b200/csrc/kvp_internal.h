@@ -173,7 +173,9 @@ struct kvp_ctx {
     int32_t sm_count = 148;
     int32_t split_target_ctas = 0, force_splits = 0;
     // optional CUDA-event timing of the attention (0) and gather (1) kernels, for roofline reports
-    bool time_kernels = false;
+    int32_t time_kernels = 0;             // 0: off; p >= 1: every p-th attention / gather kernel is bracketed by events
+    int32_t tev_seen[2] = {0, 0};
+    bool tev_open[2] = {false, false};
     std::vector<cudaEvent_t> tev[2][2];
     int32_t tev_n[2] = {0, 0};
     int32_t last_kind = -1, last_ctas = 0, last_splits = 0, last_launches = 0;
