@@ -211,6 +211,23 @@ KVP_API int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
                           const void *k_new, const void *v_new, int32_t q_len, uint32_t flags,
                           void *out, float *lse, void *stream);
 
+/*
+ * The same for a batch whose requests bring query chunks of different lengths (a serving batch rarely has equal
+ * ones; the paper's Section 3.2 is per request).  q, k_new, v_new, out, lse have the layout of kvp_query_prefill
+ * with q_len_max as the token stride; request b uses its first q_lens[b] tokens (1 <= q_lens[b] <= q_len_max).
+ * Rows of out / lse beyond a request's length are not written; the padding rows of q, k_new, v_new are never
+ * used in a result but are read, so they must hold finite numbers (zeros will do).
+ *   q_lens   host [batch]
+ * Runs on the two-stream tcgen05 kernel with its own append only (bf16, head_dim 128, sm_100a; 16-byte aligned
+ * k_new / v_new): KVP_ERR_UNSUPPORTED otherwise; no flags.  The appended rows differ per request, so this
+ * layer of the assembly cannot be continued (KVP_CONTINUE), exported with query rows or given to
+ * kvp_segment_mass afterwards.
+ * Errors: as kvp_query_prefill, INVALID (a length outside [1, q_len_max]).
+ */
+KVP_API int32_t kvp_query_prefill_ragged(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
+                                 const void *v_new, int32_t q_len_max, const int32_t *q_lens, void *out, float *lse,
+                                 void *stream);
+
 /* ---- inspection helpers (not on the hot path) -------------------------------------------------- */
 
 /*

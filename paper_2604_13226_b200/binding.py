@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         "kvp_register_adapter": (i32, [vp, vp, vp, i32, i32, vp, vp, i32, i32, vp, pi32]),
         "kvp_assemble": (i32, [vp, i32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
         "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
+        "kvp_query_prefill_ragged": (i32, [vp, i32, i32, vp, vp, vp, i32, pi32, vp, vp, vp]),
         "kvp_export_plan": (i32, [vp, i32, i32, pi32, pi32, pi32, pi32]),
         "kvp_export_cache": (i32, [vp, i32, i32, i32, i32, vp, vp, i32, vp]),
         "kvp_export_schedule": (i32, [vp, i32, i32, pi32, i32, pi32, i32, pi32, i32, pi32]),
@@ -92,7 +93,7 @@ def lib() -> ctypes.CDLL:
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_packet_host", "kvp_evict_packet",
-            "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill",
+            "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill", "kvp_query_prefill_ragged",
             "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_segment_mass", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
@@ -238,6 +239,13 @@ class Context:
                       flags: int = 0, stream=None):
         self._check(self._L.kvp_query_prefill(self._h, assembly_id, layer, _ptr(q), _ptr(k_new), _ptr(v_new), q_len,
                                               flags, _ptr(out), _ptr(lse), self._stream(stream)))
+
+    def query_prefill_ragged(self, assembly_id: int, layer: int, q, k_new, v_new, q_len_max: int, q_lens: Sequence[int],
+                             out, lse=None, stream=None):
+        """Per-request query lengths; the tensors are padded to q_len_max tokens per request."""
+        self._check(self._L.kvp_query_prefill_ragged(self._h, assembly_id, layer, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                                     q_len_max, _i32_array(list(q_lens)), _ptr(out), _ptr(lse),
+                                                     self._stream(stream)))
 
     # -- helpers ---------------------------------------------------------------------------------
     def export_plan(self, assembly_id: int, b: int):

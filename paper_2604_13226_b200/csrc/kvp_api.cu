@@ -213,22 +213,28 @@ struct schedule_t {
     int32_t n_ctas = 0, n_slots = 0, max_pieces = 1;
 };
 
-int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int q_len, int q_pos0, schedule_t &out)
+// q_lens: nullptr, or one query length per request (<= q_len, the stride of the padded tensors); a request's
+// work records and merge items then carry its own length.
+int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int q_len, int q_pos0, const int32_t *q_lens,
+                      schedule_t &out)
 {
     const kvp_shape &sh = ctx->shape;
-    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces; };
+    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces, q_len; };
     std::vector<unit_t> units;
-    const int n_rows = sh.group * q_len;
+    const int max_rows = sh.group * q_len;
     int64_t total = 0;
     // Row blocks outermost: the units of one (request, kv head) - which stream the same K/V - then lie a
     // whole number of CTA shares apart on the line (when their count divides the CTA count), so the CTAs
     // that hold them reach the same key tiles at the same time and all but the first find them in L2.
-    for (int row_base = 0; row_base < n_rows; row_base += 2 * KVP_TILE_ROWS)
+    for (int row_base = 0; row_base < max_rows; row_base += 2 * KVP_TILE_ROWS)
         for (int b = 0; b < as.batch; ++b) {
             const kvp_item &item = as.items[(as.item_stride ? layer * as.item_stride : 0) + b];
             const int n_prefix = item.tile_end - item.tile_begin;
+            const int n_rows = sh.group * (q_lens ? q_lens[b] : q_len);
+            if (row_base >= n_rows) continue;
             for (int hk = 0; hk < sh.n_kv_heads; ++hk) {
                 unit_t u;
+                u.q_len = q_lens ? q_lens[b] : 0;
                 u.b = b; u.hk = hk; u.row_base = row_base;
                 u.mode = (n_rows - row_base <= KVP_TILE_ROWS) ? 1 : 0;
                 const int last = std::min(n_rows - 1, row_base + (u.mode ? 1 : 2) * KVP_TILE_ROWS - 1);
@@ -338,7 +344,8 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
             const int32_t hi = (u == z.u) ? z.t : units[u].n_all;
             if (hi <= lo) continue;
             kvp_work w;
-            w.b = units[u].b; w.hk = units[u].hk; w.row_base = units[u].row_base; w.mode = units[u].mode;
+            w.b = units[u].b; w.hk = units[u].hk; w.row_base = units[u].row_base;
+            w.mode = units[u].mode | (units[u].q_len << 8);       // a request's own query length rides in the upper bits
             w.tile_lo = lo; w.n_tiles = hi - lo; w.slot0 = w.slot1 = -1;
             rec.ws.push_back(w);
             rec.unit.push_back(u);
@@ -385,6 +392,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
         kvp_merge_item m;
         memset(&m, 0, sizeof m);
         m.b = u.b; m.hk = u.hk; m.row_base = u.row_base; m.slot0 = base; m.n_slots = u.n_pieces;
+        m.pad[0] = u.q_len;
         merges.push_back(m);
         n_slots += u.n_pieces;
         if (u.mode == 0) {
@@ -405,10 +413,11 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     return KVP_OK;
 }
 
-int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer, int q_len, int q_pos0, cudaStream_t st)
+int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer, int q_len, int q_pos0, const int32_t *q_lens,
+                       cudaStream_t st)
 {
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, as, layer, q_len, q_pos0, sc);
+    const int32_t rc = plan_schedule(ctx, as, layer, q_len, q_pos0, q_lens, sc);
     if (rc != KVP_OK) return rc;
     const std::vector<int32_t> &cta_begin = sc.cta_begin;
     const std::vector<kvp_work> &works = sc.works;
@@ -431,6 +440,7 @@ int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer,
     KVP_CUDA(ctx, cudaEventRecord(ctx->sched_event[slot], st));
     kvp_assembly_host::sched_state &ss = as.sched[li];
     ss.q_len = q_len;
+    ss.q_lens.assign(q_lens ? q_lens : nullptr, q_lens ? q_lens + as.batch : nullptr);
     ss.q_pos0 = q_pos0;
     ss.ctas = n_ctas;
     ss.works = (int32_t)works.size();
@@ -1008,6 +1018,8 @@ int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_cache: unknown assembly %d", assembly_id);
     const kvp_assembly_host &as = ctx->slots[slot];
     if (as.item_stride) return fail(ctx, KVP_ERR_UNSUPPORTED, "export_cache: the assembly uses compressed packets");
+    if (as.ragged && n_query_rows > 0)
+        return fail(ctx, KVP_ERR_UNSUPPORTED, "export_cache: query rows after kvp_query_prefill_ragged differ per request");
     if (b < 0 || b >= as.batch || layer < 0 || layer >= ctx->cfg.n_layers || !k_out || !v_out || n_query_rows < 0 ||
         n_query_rows > ctx->cfg.max_query_tokens)
         return fail(ctx, KVP_ERR_INVALID, "export_cache: bad arguments");
@@ -1019,8 +1031,9 @@ int32_t kvp_export_cache(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, int32
     return KVP_OK;
 }
 
-int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
-                          const void *v_new, int32_t q_len, uint32_t flags, void *out, float *lse, void *stream)
+static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
+                                  const void *v_new, int32_t q_len, const int32_t *q_lens, uint32_t flags, void *out,
+                                  float *lse, void *stream)
 {
     if (!ctx) return KVP_ERR_INVALID;
     if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "query_prefill: host-only context has no device to run on");
@@ -1045,6 +1058,7 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
 
     int launches = 0;
     const bool fast = ctx->have_tma && !(flags & KVP_FORCE_SIMPLE);
+    if (q_lens && !fast) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill_ragged: needs the tcgen05 kernel (bf16, head_dim 128, sm_100)");
     // plain prefill on the two-stream kernel: it reads the query block's K/V from k_new / v_new and appends them itself
     kvp_attn2_args a;
     a.tail_direct = 0;
@@ -1053,6 +1067,8 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_knew, k_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch) &&
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_vnew, v_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch))
         a.tail_direct = 1;
+    if (q_lens && !a.tail_direct)
+        return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill_ragged: needs the tcgen05 kernel with its own append (bf16, head_dim 128, 16-byte aligned k_new / v_new)");
     if (!a.tail_direct) {
         KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q_pos0, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
                                         layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
@@ -1060,7 +1076,8 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     }
     const void *q_used = rope_query ? (const void *)ctx->q_scratch : q;
     as.last_q_len = q_len;
-    as.appended[layer] = q_pos0 + q_len;
+    as.appended[layer] = q_lens ? 0 : q_pos0 + q_len;       // after a ragged call the rows behind the prefixes differ per request
+    if (q_lens) as.ragged = true;
 
     int32_t ctas = 0, splits = 1;
     if (!fast) {
@@ -1073,8 +1090,11 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     } else if (ctx->kernel_variant == 0) {
         const int li = as.item_stride ? layer : 0;
         if (as.sched.empty()) as.sched.resize(as.item_stride ? ctx->cfg.n_layers : 1);
-        if (as.sched[li].q_len != q_len || as.sched[li].q_pos0 != q_pos0 || as.sched[li].ctas == 0) {
-            const int32_t rc = build_schedule(ctx, as, slot, layer, q_len, q_pos0, st);
+        const bool same_lens = q_lens ? (as.sched[li].q_lens.size() == (size_t)as.batch &&
+                                          std::equal(q_lens, q_lens + as.batch, as.sched[li].q_lens.begin()))
+                                       : as.sched[li].q_lens.empty();
+        if (as.sched[li].q_len != q_len || as.sched[li].q_pos0 != q_pos0 || as.sched[li].ctas == 0 || !same_lens) {
+            const int32_t rc = build_schedule(ctx, as, slot, layer, q_len, q_pos0, q_lens, st);
             if (rc != KVP_OK) return rc;
         }
         const kvp_assembly_host::sched_state &ss = as.sched[li];
@@ -1154,6 +1174,27 @@ int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, cons
     return KVP_OK;
 }
 
+int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
+                          const void *v_new, int32_t q_len, uint32_t flags, void *out, float *lse, void *stream)
+{
+    return query_prefill_impl(ctx, assembly_id, layer, q, k_new, v_new, q_len, nullptr, flags, out, lse, stream);
+}
+
+int32_t kvp_query_prefill_ragged(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const void *k_new,
+                                 const void *v_new, int32_t q_len_max, const int32_t *q_lens, void *out, float *lse,
+                                 void *stream)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!q_lens) return fail(ctx, KVP_ERR_INVALID, "query_prefill_ragged: q_lens is null");
+    const int slot = find_slot(ctx, assembly_id);
+    if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "query_prefill_ragged: unknown assembly %d", assembly_id);
+    for (int b = 0; b < ctx->slots[slot].batch; ++b)
+        if (q_lens[b] < 1 || q_lens[b] > q_len_max)
+            return fail(ctx, KVP_ERR_INVALID, "query_prefill_ragged: q_lens[%d] = %d outside [1, %d]", b, q_lens[b], q_len_max);
+    if (ctx->kernel_variant != 0) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill_ragged: two-stream kernel only");
+    return query_prefill_impl(ctx, assembly_id, layer, q, k_new, v_new, q_len_max, q_lens, 0, out, lse, stream);
+}
+
 int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const float *lse,
                          int32_t q_len, uint32_t flags, float *mass, int32_t n_cols, void *stream)
 {
@@ -1212,7 +1253,7 @@ int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, in
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_schedule: unknown assembly %d", assembly_id);
     if (q_len <= 0 || q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_INVALID, "export_schedule: bad q_len");
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], 0, q_len, 0, sc);
+    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], 0, q_len, 0, nullptr, sc);
     if (rc != KVP_OK) return rc;
     counts[0] = sc.n_ctas;
     counts[1] = (int32_t)sc.works.size();

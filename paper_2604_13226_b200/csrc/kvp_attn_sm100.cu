@@ -281,6 +281,7 @@ struct Work {
     int b, hk, row_base, mode, lo, n, slot0, slot1;
     int n_tail, tile_begin, tail_row0, plane;
     int steps0, steps1;
+    int q_len;                 // query tokens of this request (the call's q_len unless the work record carries its own)
 };
 
 __device__ __forceinline__ Work load_work(const Params &p, int wi)
@@ -288,13 +289,14 @@ __device__ __forceinline__ Work load_work(const Params &p, int wi)
     const int4 *w4 = reinterpret_cast<const int4 *>(p.works + wi);
     const int4 a = __ldg(w4), c = __ldg(w4 + 1);
     Work w;
-    w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w;
+    w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w & 0xff;
+    w.q_len = (a.w >> 8) ? (a.w >> 8) : p.q_len;
     w.lo = c.x; w.n = c.y; w.slot0 = c.z; w.slot1 = c.w;
     const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + p.layer * p.plan.item_stride + w.b);
     const int4 ia = __ldg(i4), ib = __ldg(i4 + 1);          // prefix_len, tile_begin, tile_end, seg_begin | seg_end, tail_row0, ..
     w.tile_begin = ia.y;
     w.tail_row0 = ib.y;
-    const int n_rows = p.group * p.q_len;
+    const int n_rows = p.group * w.q_len;
     const int last = min(n_rows - 1, w.row_base + (w.mode ? KVP_TILE_ROWS : 2 * KVP_TILE_ROWS) - 1);
     w.n_tail = (p.q_pos0 + last / p.group) / KVP_TILE_KEYS + 1;
     w.plane = p.layer * p.n_kv + w.hk;
@@ -313,7 +315,7 @@ __device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
     Tile t;
     if (j < w.n_tail) {
         t.row0 = p.tail_direct ? j * KVP_TILE_KEYS : w.tail_row0 + j * KVP_TILE_KEYS;
-        t.n_keys = min(KVP_TILE_KEYS, p.q_pos0 + p.q_len - j * KVP_TILE_KEYS);
+        t.n_keys = min(KVP_TILE_KEYS, p.q_pos0 + w.q_len - j * KVP_TILE_KEYS);
         t.src = p.tail_direct ? 2 : 1;               // 2: rows of the caller's k_new / v_new, by query token
         t.rope = 0;
         t.qoff = j * KVP_TILE_KEYS;
@@ -534,10 +536,10 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
         const Work w = load_work(p, wi);
         const int steps = S == 0 ? w.steps0 : w.steps1;
         if (steps == 0) continue;
-        const int n_rows = p.group * p.q_len;
+        const int n_rows = p.group * w.q_len;
         const int r = w.row_base + (w.mode == 0 ? S * KVP_TILE_ROWS : 0) + t;
         const bool valid = r < n_rows;
-        const int qi = valid ? r / p.group : p.q_len - 1;
+        const int qi = valid ? r / p.group : w.q_len - 1;
         const int h = w.hk * p.group + (valid ? r % p.group : 0);
 
         float m_ref = -1e30f, l = 0.f;
@@ -684,7 +686,7 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
     bool ok = true;
     for (int wi = c.item_begin; wi < c.item_end && ok; ++wi) {
         const Work w = load_work(p, wi);
-        const int n_rows = p.group * p.q_len;
+        const int n_rows = p.group * w.q_len;
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
         auto produce = [&](int s, int rope, uint32_t &nEp) {
@@ -725,7 +727,7 @@ __device__ __forceinline__ void append_role(const Params &p, const Cta &c, const
     for (int wi = c.item_begin; wi < c.item_end; ++wi) {
         const Work w = load_work(p, wi);
         if (w.lo != 0 || w.row_base != 0) continue;
-        for (int i = t; i < p.q_len * 16; i += 64) {            // 16-byte words of the rows of this kv head
+        for (int i = t; i < w.q_len * 16; i += 64) {            // 16-byte words of the rows of this kv head
             const int row = i >> 4, c4 = i & 15;
             const long long src = (((long long)w.b * p.q_len + row) * p.n_kv + w.hk) * 16 + c4;
             const long long dst = ((long long)w.plane * p.ws_rows + w.tail_row0 + row) * 16 + c4;
@@ -1107,7 +1109,7 @@ merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q,
     const kvp_merge_item mi = merges[blockIdx.x];
     const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5;
     const int row = blockIdx.y * 32 + lane;                     // row of the 128-row query tile
-    const int n_rows = group * q_len;
+    const int n_rows = group * (mi.pad[0] ? mi.pad[0] : q_len);         // q_len stays the stride of the padded tensors
     const float c2 = scale * 1.4426950408889634f;
     const float4 *po = reinterpret_cast<const float4 *>(part_o);
     float M = -INFINITY;

@@ -71,7 +71,7 @@ struct kvp_merge_item {        // 128 packed rows whose result is spread over n_
     int32_t b, hk;
     int32_t row_base;
     int32_t slot0, n_slots;
-    int32_t pad[3];
+    int32_t pad[3];            // pad[0]: the request's own query length (0: the call's q_len)
 };
 
 // Offsets (bytes) of the arrays inside one plan blob; identical on host and device.
@@ -117,10 +117,11 @@ struct kvp_assembly_host {
     int32_t item_stride = 0;               // batch when the assembly has per-layer tile lists (compressed packets)
     int32_t last_q_len = 0;
     std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
+    bool ragged = false;                   // a kvp_query_prefill_ragged call has appended a different number of rows per request
     bool waits_loads = false;              // uses packets that came from host memory: wait for the layer's load event
     // work lists of the two-stream kernel (one, or one per layer when the tile lists differ per layer), each
     // built for q_len query tokens at offset q_pos0 (q_len 0 = none yet)
-    struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; };
+    struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; std::vector<int32_t> q_lens; };
     std::vector<sched_state> sched;
 };
 
