@@ -572,7 +572,7 @@ def main():
                         "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": peaks["source"]}
             roof.update({"kernel": "attn_sm100_kernel", "launches_timed": len(attn_ms), "avg_launch_ms": a_ms,
                          "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
-                         "attn_share_of_step": sum(attn_ms) / ms_total,
+                         "attn_share_of_step": a_ms * L * args.steps / ms_total,     # every launch counted at the sampled mean
                          "gather_avg_ms": statistics.mean(gather_ms) if gather_ms else None})
         else:
             roof = None
