@@ -425,9 +425,8 @@ struct Cta {
 };
 
 // ---- softmax / correction / epilogue of stream S -------------------------------------------------------
-// One thread per query row.  S is read from TMEM in 32-column chunks, twice (row max, then exponentials);
-// the chunk loops are rolled and shared by both streams so that the code stays resident in the
-// instruction cache; the next chunk is requested before the current one is processed.
+// One thread per query row.  S is read from TMEM in 32-column chunks, once; the chunk loop is rolled and
+// shared by both streams so that the code stays resident in the instruction cache.
 __device__ __forceinline__ float chunk_max(const uint32_t *v, float m)
 {
     float m0 = m, m1 = m;
@@ -556,7 +555,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
 
             const bool full = (tl.n_keys == KVP_TILE_KEYS) && (tl.qoff < 0);
             const int lim = tl.qoff < 0 ? tl.n_keys : min(tl.n_keys, p.q_pos0 + qi - tl.qoff + 1);       // visible keys: [0, lim)
-            uint32_t va[32], vb[32];
+            uint32_t va[32];
 
             // One pass over S: the exponentials use the reference max carried over from earlier tiles; each
             // 32-column chunk's own max is checked first, and only if it exceeds the reference by more than
@@ -572,8 +571,6 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
                 if (__any_sync(0xffffffffu, need)) {
                     const float m_new = need ? cm : m_ref;
                     const float alpha = need ? ex2((m_ref - m_new) * c2) : 1.f;
-                    tc_wait_ld();                          // the other buffer's chunk may still be in flight
-                    landed32(v == va ? vb : va);
                     rescale_row(s_addr, o_addr, alpha, ch, k > 0);
                     l *= alpha;
                     m_ref = m_new;
