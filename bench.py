@@ -62,7 +62,7 @@ def make_spec(name: str, seed: int):
 
 def algorithmic_work(spec):
     """Per layer: flops = 4 d Hq Lq (P + (Lq+1)/2) per request; bytes = prefix K,V once + Q, O, K_new,
-    V_new read and appended ('algorithmic work')."""
+    V_new read once and the appended rows written once (every byte the step must move, moved once)."""
     s = spec.shape
     d, Hq, Hkv, e, Lq = s.head_dim, s.n_q_heads, s.n_kv_heads, s.elem_bytes, spec.q_len
     flops = bytes_ = 0.0
