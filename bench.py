@@ -44,12 +44,39 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# NVIDIA's nominal B200 figures (dense bf16; HBM3e), for the "of nominal" fractions
+NOMINAL_TFLOPS, NOMINAL_GBS, N_SMS = 2250.0, 8000.0, 148
+
+
+def tensor_fractions(tflops: float, peaks, region_s: float, clocks):
+    """One achieved bf16 rate against every denominator, and the headline fraction by a stated rule: the burst
+    GEMM peak when the timed region is shorter than one second or the SM clock sampled during it stayed at
+    >= 0.9 of its maximum (the conditions the burst peak was measured under), the sustained peak otherwise."""
+    sm = (clocks or {}).get("sm_mhz")
+    mx = (clocks or {}).get("sm_max_mhz")
+    burst = region_s < 1.0 or (sm is not None and mx and sm >= 0.9 * mx)
+    out = {"frac_burst": tflops / peaks["bf16_tflops"], "frac_sustained": tflops / peaks["bf16_tflops_sustained"],
+           "frac_nominal": tflops / NOMINAL_TFLOPS,
+           "peak_burst": peaks["bf16_tflops"], "peak_sustained": peaks["bf16_tflops_sustained"], "peak_nominal": NOMINAL_TFLOPS,
+           "headline_peak": "burst" if burst else "sustained",
+           "headline_rule": "burst if timed region < 1 s or median SM clock >= 0.9 max, else sustained",
+           "rule_inputs": {"timed_region_s": region_s, "sm_mhz_median": sm, "sm_max_mhz": mx}}
+    if sm:
+        # clock-normalised: flop per SM cycle (the tensor pipe's ceiling is 8192 dense bf16 flop per SM cycle)
+        out["flop_per_sm_cycle"] = tflops * 1e12 / (sm * 1e6 * N_SMS)
+    return out, (peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"])
+
+
 def make_spec(name: str, seed: int):
     from paper_2604_13226_b200 import inputs as gen
     if name == "config3":
         return gen.spec_config3(seed=seed)
     if name == "config4":
         return gen.spec_config4(seed=seed)
+    if name == "config4_layer":                      # one layer of the Qwen2.5-7B stack: same requests, same raggedness
+        s = gen.spec_config4(seed=seed, n_layers=1)
+        s.name = "config4_layer"
+        return s
     if name == "config2":
         s = gen.spec_config3(seed=seed, n_layers=1, batch=1, pool=5, per_item=5, doc_len=512, q_len=64)
         s.name = "config2"
@@ -100,61 +127,92 @@ def job_tokens_per_s(spec, world: int, ms_step: float) -> float:
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """nvidia-smi clock / throttle-reason samples, every 20 ms, taken for as long as the sampler runs; every
+    sample carries nvidia-smi's own timestamp, so any timed region gets the record of exactly its samples."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, index: int):
-        self.index = index
+    def __init__(self, index: int, period_ms: int = 20):
+        self.index, self.period_ms = index, period_ms
         self.proc = None
+        self.samples = []                      # (epoch seconds, sm MHz, max MHz, watts, set of active reasons)
+        self._thread = None
+
+    def _read(self):
+        import datetime
+        for line in self.proc.stdout:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                t = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                self.samples.append((t, float(f[1]), float(f[2]), float(f[3]),
+                                     {n for n, v in zip(self.NAMES, f[4:8]) if v.lower().startswith("active")}))
+            except ValueError:
+                continue
 
     def start(self):
+        import threading
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "--format=csv,noheader,nounits", "-lms", str(self.period_ms)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
+            self._thread = threading.Thread(target=self._read, daemon=True)
+            self._thread.start()
         except Exception:
             self.proc = None
 
+    @staticmethod
+    def now() -> float:
+        return time.time()
+
     def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+            return
+        time.sleep(0.1)
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-            out = ""
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        # keep samples taken under load (upper half) for the median
-        sm_sorted = sorted(sm)
-        load = sm_sorted[len(sm_sorted) // 2:] if sm_sorted else []
-        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        if self._thread is not None:
+            self._thread.join(timeout=5)
+
+    def window(self, t0: float, t1: float):
+        """Record of the samples stamped inside [t0, t1] (widened to the nearest sample on either side when the
+        region is shorter than the sampling period)."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        time.sleep(3 * self.period_ms / 1000.0)           # let the samples of the region's end arrive
+        inside = [x for x in self.samples if t0 <= x[0] <= t1]
+        if len(inside) < 2:
+            mid = 0.5 * (t0 + t1)
+            inside = sorted(self.samples, key=lambda x: abs(x[0] - mid))[:2]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"], "samples": 0}
+        reasons = set()
+        for x in inside:
+            reasons |= x[4]
+        return {"sm_mhz": statistics.median(x[1] for x in inside), "sm_mhz_min": min(x[1] for x in inside),
+                "sm_max_mhz": max(x[2] for x in inside), "power_w_max": max(x[3] for x in inside),
+                "reasons": sorted(reasons), "samples": len(inside), "period_ms": self.period_ms}
 
 
 # ---------------------------------------------------------------------------------------------------
 # oracle timing (cpu_baseline leg and the --impl reference arm)
 # ---------------------------------------------------------------------------------------------------
 
-def oracle_sample(spec, wl, n_tokens: int = 0):
-    """Time the fp64 oracle, as it stands, on layer 0 of every request: composition + re-basing of the
-    whole prefix, then attention for every head of `n_tokens` query tokens (0 = all).  Returns the
-    job-level rate it implies: query tokens/s through the full stack = batch*q_len / (L * sum_b t_b)."""
+ORACLE_TOKENS = 32          # query tokens per request the oracle is timed on (evenly spaced over the chunk)
+
+
+def oracle_sample(spec, wl, n_tokens: int = ORACLE_TOKENS):
+    """Time the fp64 oracle, as it stands, on layer 0 of every request: composition + re-basing of the whole
+    prefix and the widening / concatenation of its inputs (a fixed cost per request and layer), then attention
+    for every head of `n_tokens` query tokens spread evenly over the chunk (0 = all).  Only the attention time is
+    scaled to the full chunk (work per row is the same to within q_len / prefix).  Returns the job-level rate it
+    implies: query tokens/s through the full stack = batch*q_len / (L * sum_b t_b).  `cpu_baseline` and the
+    reference arm both call this with the default sample."""
     from oracle import reference as orc
     s = spec.shape
     ad = wl.adapter_host()
@@ -171,30 +229,47 @@ def oracle_sample(spec, wl, n_tokens: int = 0):
         st.register_packet(n, 0, (lambda layer, pid=pid: cached[pid]))
     st.register_adapter(ad.n_header, 0, ad.n_trailer, 0, (lambda layer: (ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0])))
     toks = list(range(spec.q_len))
-    if n_tokens > 0:
-        pick = sorted(set([0, 1, 63, 64, 127, 128, spec.q_len - 1]) & set(toks))
-        toks = pick[:n_tokens]
+    if 0 < n_tokens < spec.q_len:
+        toks = sorted({int(round(i * (spec.q_len - 1) / (n_tokens - 1))) for i in range(n_tokens)}) if n_tokens > 1 else [spec.q_len - 1]
     rows = [(h, i) for i in toks for h in range(s.n_q_heads)]
-    t_total = t_comp = t_att = 0.0
+    t_total = t_fixed = t_att = 0.0
     for b in range(spec.batch):
         t0 = time.perf_counter()
         plan = orc.compose(st, spec.items[b], spec.rebase)
         Kp, Vp, _ = orc.composed_kv(st, plan, 0, f, s.rope_pairing)
-        t1 = time.perf_counter()
         Q = orc.widen(q[b], s.dtype)
         K = np.concatenate([Kp, orc.widen(kn[b], s.dtype)])
         V = np.concatenate([Vp, orc.widen(vn[b], s.dtype)])
+        t1 = time.perf_counter()
         orc.attention_rows(K, V, Q, plan.prefix_len, 1.0 / np.sqrt(s.head_dim), rows)
         t2 = time.perf_counter()
-        t_comp += t1 - t0
+        t_fixed += t1 - t0
         t_att += t2 - t1
         t_total += (t1 - t0) + (t2 - t1) / len(rows) * (spec.q_len * s.n_q_heads)
     tokens_per_s = spec.batch * spec.q_len / (s.n_layers * t_total)
     return {"value": tokens_per_s, "unit": "tokens/s", "cores": orc.threads(), "kind": "oracle",
-            "sample": f"layer 0 of all {spec.batch} requests: compose + re-base of the prefix ({t_comp:.2f} s) and attention "
-                      f"rows of {len(toks)} of {spec.q_len} query tokens x {s.n_q_heads} heads ({t_att:.2f} s); scaled to "
-                      f"{spec.q_len} tokens x {s.n_layers} layers",
-            "seconds": t_comp + t_att}
+            "sample": f"layer 0 of all {spec.batch} requests: compose + re-base + widening of the prefix ({t_fixed:.2f} s) and "
+                      f"attention rows of {len(toks)} of {spec.q_len} query tokens x {s.n_q_heads} heads ({t_att:.2f} s); "
+                      f"attention scaled to {spec.q_len} tokens, the sum to {s.n_layers} layers",
+            "seconds": t_fixed + t_att}
+
+
+def prefill_flags(spec) -> int:
+    """Workloads with x8 outlier channels are run the way their parity test runs them: KVP_PRECISE_QK."""
+    from paper_2604_13226_b200 import binding as kvp
+    return kvp.PRECISE_QK if getattr(spec, "outlier_channels", 0) else 0
+
+
+def workload_config(spec, materialize: bool, bytes_per_layer: float):
+    """The `config` object of the JSON line: the workload, named the same way by both arms."""
+    s = spec.shape
+    return {"workload": spec.name, "layers": s.n_layers, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
+            "head_dim": s.head_dim, "batch_per_gpu": spec.batch, "q_len": spec.q_len,
+            "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)], "rope_theta": s.rope_theta,
+            "mode": "materialised cache" if materialize else "fused in place (adapters staged)",
+            "qk": "precise (KVP_PRECISE_QK)" if prefill_flags(spec) else "plain",
+            "l2": "inputs larger than L2: every layer reads %.0f MB of distinct K/V" % (bytes_per_layer / 1e6),
+            "sharding": "requests sharded across ranks, no collective"}
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -207,7 +282,17 @@ def flush_l2(torch, dev, buf=[None]):
     buf[0].zero_()
 
 
-def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peaks, device: int):
+def point_fractions(res, flops, bytes_, ms, peaks, clocks, region_s):
+    """Rates of one timed kernel against the measured (burst / sustained) and nominal peaks."""
+    tf = flops / ms / 1e9
+    fr, _ = tensor_fractions(tf, peaks, region_s, clocks)
+    res.update({"frac_tensor_burst": fr["frac_burst"], "frac_tensor_sustained": fr["frac_sustained"],
+                "frac_tensor_nominal": fr["frac_nominal"], "flop_per_sm_cycle": fr.get("flop_per_sm_cycle"),
+                "frac_hbm": bytes_ / ms / 1e6 / peaks["hbm_gbs"], "frac_hbm_nominal": bytes_ / ms / 1e6 / NOMINAL_GBS,
+                "clocks": clocks})
+
+
+def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peaks, device: int, sampler=None):
     """ms of one layer's attention kernel (CUDA events inside the library) and of the gather kernel."""
     import torch
     from paper_2604_13226_b200 import binding as kvp, inputs as gen
@@ -218,17 +303,20 @@ def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peak
     sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 1)
     dev = torch.device(f"cuda:{device}")
     qkv = sess.query_tensors(0)
+    flags = prefill_flags(spec)
     att, gat = [], []
+    t0 = ClockSampler.now()
     for it in range(iters + 3):
         flush_l2(torch, dev)
         sess.assemble()
         flush_l2(torch, dev)
-        sess.prefill(0, qkv=qkv, want_lse=False)
+        sess.prefill(0, flags, qkv=qkv, want_lse=False)
         torch.cuda.synchronize(dev)
         a, g = sess.ctx.kernel_times(0), sess.ctx.kernel_times(1)
         if it >= 3:
             att += a
             gat += g
+    clocks = sampler.window(t0, ClockSampler.now()) if sampler is not None else None
     launch = sess.ctx.last_launch()
     assert sess.ctx.status_word() == 0
     flops, bytes_ = algorithmic_work(spec)
@@ -245,15 +333,15 @@ def measure_point(spec_name: str, seed: int, iters: int, materialize: bool, peak
     del sess, wl
     torch.cuda.empty_cache()
     res = {"workload": spec.name, "attn_ms": ms_a, "attn_tflops": flops / ms_a / 1e9, "attn_gbs": bytes_ / ms_a / 1e6,
-           "frac_tensor_sustained": flops / ms_a / 1e9 / peaks["bf16_tflops_sustained"],
-           "frac_hbm": bytes_ / ms_a / 1e6 / peaks["hbm_gbs"], "launch": launch, "l2": "flushed between iterations"}
+           "launch": launch, "l2": "flushed between iterations", "qk": "precise (KVP_PRECISE_QK)" if flags else "plain"}
+    point_fractions(res, flops, bytes_, ms_a, peaks, clocks, ms_a * 1e-3)      # launches timed one at a time: burst conditions
     if ms_g:
         res.update({"gather_ms": ms_g, "gather_gbs": gather_bytes / ms_g / 1e6,
                     "gather_frac_hbm": gather_bytes / ms_g / 1e6 / peaks["hbm_gbs"], "gather_bytes": gather_bytes})
     return res
 
 
-def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: float = 0.5):
+def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: float = 0.5, sampler=None):
     """One layer of the config-3 shape (4 requests x 10 x 1024-token packets, 128 query tokens) with every
     document pruned to about `keep` of its tokens, a different subset per kv head: attention kernel time,
     and the rates counted on the keys that are actually held."""
@@ -269,6 +357,7 @@ def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: fl
     sess.assemble()
     qkv = sess.query_tensors(0)
     att = []
+    t0 = ClockSampler.now()
     for it in range(iters + 3):
         flush_l2(torch, dev)
         sess.prefill(0, qkv=qkv, want_lse=False)
@@ -276,6 +365,7 @@ def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: fl
         a = sess.ctx.kernel_times(0)
         if it >= 3:
             att += a
+    clocks = sampler.window(t0, ClockSampler.now()) if sampler is not None else None
     assert sess.ctx.status_word() == 0
     launch = sess.ctx.last_launch()
     d, g, Lq = shape.head_dim, shape.group, 128
@@ -292,10 +382,11 @@ def measure_compressed_point(seed: int, iters: int, peaks, device: int, keep: fl
     sess.close()
     del sess, wl
     torch.cuda.empty_cache()
-    return {"workload": "config3 shape, one layer, documents pruned per kv head", "kept_fraction": held / total, "attn_ms": ms,
-            "attn_tflops_on_held_keys": flops / ms / 1e9, "attn_gbs_on_held_keys": bytes_ / ms / 1e6,
-            "frac_tensor_sustained": flops / ms / 1e9 / peaks["bf16_tflops_sustained"], "launch": launch,
-            "l2": "flushed between iterations"}
+    res = {"workload": "config3 shape, one layer, documents pruned per kv head", "kept_fraction": held / total, "attn_ms": ms,
+           "attn_tflops_on_held_keys": flops / ms / 1e9, "attn_gbs_on_held_keys": bytes_ / ms / 1e6, "launch": launch,
+           "l2": "flushed between iterations"}
+    point_fractions(res, flops, bytes_, ms, peaks, clocks, ms * 1e-3)
+    return res
 
 
 def measure_host_packets_point(seed: int, iters: int, device: int, n_layers: int = 8):
@@ -385,13 +476,16 @@ def main():
         if rank != 0:
             return
         assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+        sweep_sampler = ClockSampler(local_rank)
+        sweep_sampler.start()
         for n in (2, 4, 8, 16, 32, 64):
             for ql in (16, 64, 256, 1024):
                 for b in (1, 4, 16):
-                    r = measure_point(f"config5:{n}:{ql}:{b}", args.seed, 5, False, peaks, local_rank)
+                    r = measure_point(f"config5:{n}:{ql}:{b}", args.seed, 5, False, peaks, local_rank, sweep_sampler)
                     r.pop("gather_ms", None); r.pop("gather_gbs", None); r.pop("gather_frac_hbm", None); r.pop("gather_bytes", None)
                     r.update({"packets": n, "q_len": ql, "batch": b, "bound": "tensor" if 4 * ql >= 247 else "hbm"})
                     print(json.dumps(r), flush=True)
+        sweep_sampler.stop()
         return
 
     if args.impl == "reference":
@@ -406,21 +500,19 @@ def main():
         for _ in range(args.warmup):
             oracle_sample(spec, wl, n_tokens=1)
         t0 = time.perf_counter()
-        vals = [oracle_sample(spec, wl, n_tokens=0 if args.steps <= 4 else 5) for _ in range(max(1, args.steps))]
+        vals = [oracle_sample(spec, wl) for _ in range(max(1, args.steps))]      # the sample cpu_baseline times
         dt = time.perf_counter() - t0
         v = statistics.median(x["value"] for x in vals)
         cb = dict(vals[-1])
         cb["value"] = v
-        s = spec.shape
+        _, bytes_ = algorithmic_work(spec)
+        cfg = workload_config(spec, args.materialize, bytes_)
+        cfg["note"] = "each step = a bounded sample of the workload run through the CPU oracle"
         print(json.dumps({
             "impl": "reference", "metric": "composed_cache_prefill_query_tokens_per_s", "value": v, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": spec.batch * spec.q_len / v * 1e3, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": spec.name, "layers": s.n_layers, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
-                       "head_dim": s.head_dim, "batch": spec.batch, "q_len": spec.q_len,
-                       "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)],
-                       "note": "each step = a bounded sample of the workload run through the CPU oracle"},
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
             "cpu_baseline": cb, "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0, "wall_s": dt}))
         return
@@ -454,8 +546,9 @@ def main():
         sess.assemble()
         for l in range(L):
             q, kn, vn = qkv[l]
-            sess.ctx.query_prefill(sess.assembly_id, l, q, kn, vn, Lq, outs[l], None, 0)
+            sess.ctx.query_prefill(sess.assembly_id, l, q, kn, vn, Lq, outs[l], None, pf_flags)
 
+    pf_flags = prefill_flags(spec)
     for _ in range(args.warmup):
         step()
     barrier()
@@ -466,14 +559,16 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        time.sleep(0.1)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_region0 = ClockSampler.now()
     ev0.record()
     for _ in range(args.steps):
         step()
     ev1.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.window(t_region0, ClockSampler.now()) if rank == 0 else None
     ms_total = ev0.elapsed_time(ev1)
     attn_ms = sess.ctx.kernel_times(0)
     gather_ms = sess.ctx.kernel_times(1)
@@ -509,7 +604,7 @@ def main():
             with torch.cuda.stream(s_run):
                 s_run.wait_event(ev_in[k])
                 s_run.wait_event(ev_out[k])                    # its previous result has left the device
-                sess.ctx.query_prefill(sess.assembly_id, l, dq[k][0], dq[k][1], dq[k][2], Lq, dout[k], None, 0)
+                sess.ctx.query_prefill(sess.assembly_id, l, dq[k][0], dq[k][1], dq[k][2], Lq, dout[k], None, pf_flags)
                 ev_run[k].record(s_run)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_run[k])
@@ -563,13 +658,15 @@ def main():
         if a_ms:
             if tensor_bound:
                 ach = flops / a_ms / 1e9
-                roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                        "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                        "peak_source": peaks["source"] + " (sustained bf16 GEMM; burst %.1f)" % peaks["bf16_tflops"]}
+                fr, peak = tensor_fractions(ach, peaks, ms_total * 1e-3, clocks)
+                roof = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                        "traffic": traffic, "peak_source": peaks["source"] + " (%s bf16 GEMM)" % fr["headline_peak"]}
+                roof.update(fr)
             else:
                 ach = bytes_ / a_ms / 1e6
                 roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": peaks["source"]}
+                        "frac": ach / peaks["hbm_gbs"], "frac_nominal": ach / NOMINAL_GBS, "peak_nominal": NOMINAL_GBS,
+                        "traffic": traffic, "peak_source": peaks["source"]}
             roof.update({"kernel": "attn_sm100_kernel", "launches_timed": len(attn_ms), "avg_launch_ms": a_ms,
                          "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": bytes_,
                          "attn_share_of_step": a_ms * L * args.steps / ms_total,     # every launch counted at the sampled mean
@@ -581,12 +678,7 @@ def main():
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32",
             "data": "synthetic",
-            "config": {"workload": spec.name, "layers": L, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
-                       "head_dim": s.head_dim, "batch_per_gpu": spec.batch, "q_len": Lq,
-                       "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)], "rope_theta": s.rope_theta,
-                       "mode": "materialised cache" if args.materialize else "fused in place (adapters staged)",
-                       "l2": "inputs larger than L2: every layer reads %.0f MB of distinct K/V" % (bytes_ / 1e6),
-                       "sharding": "requests sharded across ranks, no collective"},
+            "config": workload_config(spec, args.materialize, bytes_),
             "prefix_tokens_per_s": sum(spec.prefix_len(b) for b in range(spec.batch)) * world / (ms_step * 1e-3),
             "e2e": {"value": tokens / (ms_e2e / args.steps * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e / args.steps,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -595,17 +687,21 @@ def main():
         if not args.no_extras and world == 1:
             extras = {}
             try:
-                extras["hbm_bound_point"] = measure_point("config5:64:16:1", args.seed, 10, False, peaks, local_rank)
-                extras["gather_materialise_point"] = measure_point("config5:16:64:1", args.seed, 10, True, peaks, local_rank)
+                extras["hbm_bound_point"] = measure_point("config5:64:16:1", args.seed, 10, False, peaks, local_rank, sampler)
+                extras["gather_materialise_point"] = measure_point("config5:16:64:1", args.seed, 10, True, peaks, local_rank, sampler)
                 # the step after the prefill: one new token per request over 16 x 33,280-token composed caches
-                extras["decode_point"] = measure_point("config5:16:1:16", args.seed, 10, False, peaks, local_rank)
-                extras["compressed_point"] = measure_compressed_point(args.seed, 10, peaks, local_rank)
+                extras["decode_point"] = measure_point("config5:16:1:16", args.seed, 10, False, peaks, local_rank, sampler)
+                # one layer of the Qwen2.5-7B stack (28/4 heads, ragged prefixes, 256 query tokens, batch 8) and config 2
+                extras["config4_layer"] = measure_point("config4_layer", args.seed, 10, False, peaks, local_rank, sampler)
+                extras["config2"] = measure_point("config2", args.seed, 10, False, peaks, local_rank, sampler)
+                extras["compressed_point"] = measure_compressed_point(args.seed, 10, peaks, local_rank, sampler=sampler)
                 extras["host_packets_point"] = measure_host_packets_point(args.seed, 5, local_rank)
             except Exception as ex:                                   # extras never invalidate the main line
                 extras["error"] = repr(ex)
             line["extra_points"] = extras
             wl2 = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
             line["cpu_baseline"] = oracle_sample(spec, wl2)
+        sampler.stop()
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -55,7 +55,8 @@ enum {
 enum {
     KVP_ROPE_QUERY = 1u,      /* q and k_new are raw: rotate them at positions prefix_len[b] + i        */
     KVP_FORCE_SIMPLE = 2u,    /* use the plain fp32 CUDA-core kernel (cross-check path, any dtype)      */
-    KVP_CONTINUE = 4u         /* the q_len tokens follow the rows this layer's earlier calls appended   */
+    KVP_CONTINUE = 4u,        /* the q_len tokens follow the rows this layer's earlier calls appended   */
+    KVP_PRECISE_QK = 8u       /* tcgen05 path: carry the re-based operand of q.k in two bf16 numbers    */
 };
 
 typedef struct kvp_ctx kvp_ctx;
@@ -153,8 +154,8 @@ KVP_API int32_t kvp_evict_packet(kvp_ctx *ctx, int32_t packet_id);
  *   k, v   device; for (l, h) in that order, kept[l][h] rows of head_dim elements, the runs back to back
  *   kept   host [n_layers][n_kv_heads]
  * The packet occupies max(kept) pool rows.  Needs cfg.max_compressed > 0.  Assemblies that use a
- * compressed packet cannot be materialised (KVP_MATERIALIZE) or exported with kvp_export_cache, and run
- * on the two-stream tcgen05 kernel or the CUDA-core kernel only: those return KVP_ERR_UNSUPPORTED.
+ * compressed packet cannot be materialised (KVP_MATERIALIZE) or exported with kvp_export_cache: those
+ * return KVP_ERR_UNSUPPORTED.
  * Errors: INVALID, CAPACITY (max_packets, pool), STATE (max_compressed == 0), CUDA.
  */
 KVP_API int32_t kvp_register_packet_compressed(kvp_ctx *ctx, const void *k, const void *v, int32_t n_tokens,
@@ -199,6 +200,14 @@ KVP_API int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_of
  *   lse    device float [batch][n_q_heads][q_len] or NULL: natural-log sum of exp(scaled scores)
  * By default q and k_new are already rotated for positions prefix_len[b] + i; KVP_ROPE_QUERY makes
  * the library rotate them.
+ * KVP_PRECISE_QK: the tcgen05 kernel applies Eq. 1 to the query side of q.k (a document's keys stay as they
+ * were cached) and rounds the rotated query to bf16 once per document - the rounding any bf16 cache of
+ * re-based keys carries, 2^-9 relative per term of the dot product.  With this flag the rotated query is
+ * kept as value + rounding remainder (two bf16 numbers) and both are multiplied with the keys, which removes
+ * that rounding from the scores at 1.5x the Q.K tensor work on document tiles.  Meant for caches with
+ * outlier channels, where the plain rounding, multiplied by values of magnitude 10 and more, shows in the
+ * output.  No effect on the CUDA-core kernel (fp32 throughout) or on a materialised cache (its keys are
+ * stored re-based and rounded).
  * KVP_CONTINUE (the step after the prefill - decoding with q_len = 1 - or a prefill fed in chunks): the
  * rows appended by the earlier calls for this layer since kvp_assemble stay; with n of them, token i of
  * this call sits at position prefix_len[b] + n + i, attends to the prefix, to those n rows and to this
@@ -297,17 +306,14 @@ KVP_API int32_t kvp_last_launch(kvp_ctx *ctx, int32_t *kind, int32_t *ctas, int3
 
 /* Launch tuning (not needed for correctness).  key KVP_TUNE_SPLIT_TARGET_CTAS: the tcgen05 path
    splits each request's keys until about `value` CTAs exist (0 = default, 4 per SM);
-   key KVP_TUNE_FORCE_SPLITS: use exactly `value` key splits (0 = automatic; for the two-stream kernel only
-   1 is meaningful: no unit is split);
-   key KVP_TUNE_KERNEL_VARIANT: 0 = two-stream persistent tcgen05 kernel (default), 1 = single-tile kernel;
+   key KVP_TUNE_FORCE_SPLITS: 1 = no unit's key range is split (0 = automatic);
    key KVP_TUNE_FUSED_APPEND: 1 (default) = on the plain prefill path (no KVP_ROPE_QUERY, no KVP_CONTINUE) the
    tcgen05 kernel reads the query block's keys and values straight from k_new / v_new and appends them itself,
    0 = always run the separate append kernel first;
    key KVP_TUNE_TIME_KERNELS: value p >= 1 brackets every p-th attention kernel and every p-th gather kernel
    with CUDA events on the caller's stream (up to 4096 timed launches between two kvp_kernel_times calls; the
    events between back-to-back launches cost a little, hence the period), 0 = off. */
-enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3, KVP_TUNE_KERNEL_VARIANT = 4,
-       KVP_TUNE_FUSED_APPEND = 5 };
+enum { KVP_TUNE_SPLIT_TARGET_CTAS = 1, KVP_TUNE_FORCE_SPLITS = 2, KVP_TUNE_TIME_KERNELS = 3, KVP_TUNE_FUSED_APPEND = 5 };
 KVP_API int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value);
 
 /* Device durations, in milliseconds, of the kernels launched since the last call with this `which`
@@ -338,11 +344,14 @@ KVP_API int32_t kvp_kernel_times(kvp_ctx *ctx, int32_t which, float *ms, int32_t
  * so nothing depends on its old contents, but calls whose kernels can overlap on the GPU (different
  * streams or threads) race on it and must be serialised by the caller.
  *
- * The first call on each device looks up the array's device address (the device must be current);
- * make that first call outside any stream capture.  Two kernels are enqueued on `stream`; the call
- * does not synchronise.  No cudaMalloc/cudaFree or other allocating routine is called.
+ * The first call on each device looks up the array's device address (the device must be current) and
+ * makes the CUDA runtime load this library's kernels, which the driver may serve with allocations of
+ * its own: make one warm-up call per device while allocation is still allowed (before the heap is
+ * frozen) and outside any stream capture.  Two kernels are enqueued on `stream`; the call does not
+ * synchronise.  The library itself calls no cudaMalloc/cudaFree or other allocating routine here.
  * err (optional, err_cap bytes) receives a message on failure.
- * Errors: INVALID (null pointer, bad shape/dtype, segment outside the pool), CAPACITY, CUDA.
+ * Errors: INVALID (null or misaligned pointer, bad shape/dtype, segment outside the pool), CAPACITY
+ * (too many segments, or more rows than cache_rows or than 2^31 - 1), CUDA.
  */
 #define KVP_NOALLOC_MAX_SEGMENTS 96
 KVP_API int32_t kvp_compose_noalloc(const void *pool_k, const void *pool_v, int64_t pool_rows, int32_t n_planes,

@@ -18,8 +18,8 @@ STATUS_NAMES = {0: "KVP_OK", 1: "KVP_ERR_INVALID", 2: "KVP_ERR_CAPACITY", 3: "KV
                 4: "KVP_ERR_STATE", 5: "KVP_ERR_UNSUPPORTED", 6: "KVP_ERR_CUDA", 7: "KVP_ERR_TIMEOUT"}
 DTYPE_F32, DTYPE_BF16 = 0, 1
 REBASE, MATERIALIZE = 1, 2
-ROPE_QUERY, FORCE_SIMPLE, CONTINUE = 1, 2, 4
-TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS, TUNE_KERNEL_VARIANT, TUNE_FUSED_APPEND = 1, 2, 3, 4, 5
+ROPE_QUERY, FORCE_SIMPLE, CONTINUE, PRECISE_QK = 1, 2, 4, 8
+TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS, TUNE_FUSED_APPEND = 1, 2, 3, 5
 
 
 class KvpError(RuntimeError):

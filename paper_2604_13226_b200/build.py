@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libkvp.so")
-SOURCES = ["kvp_api.cu", "kvp_kernels.cu", "kvp_attn_sm100.cu", "kvp_attn_sm100_single.cu", "kvp_compose_noalloc.cu"]
+SOURCES = ["kvp_api.cu", "kvp_kernels.cu", "kvp_attn_sm100.cu", "kvp_compose_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -592,7 +592,7 @@ int32_t kvp_create(const kvp_config *cfg, kvp_ctx **out)
                 ok = make_tensor_map(enc, &ctx->tm_ws_k[a], ctx->slot_k[a], sh.head_dim, sh.ws_rows, planes) &&
                      make_tensor_map(enc, &ctx->tm_ws_v[a], ctx->slot_v[a], sh.head_dim, sh.ws_rows, planes);
             if (!ok) return bail(KVP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-            if (kvp_attn_sm100_prepare() != cudaSuccess || kvp_attn_sm100_single_prepare() != cudaSuccess)
+            if (kvp_attn_sm100_prepare() != cudaSuccess)
                 return bail(KVP_ERR_CUDA, "tcgen05 kernel attribute setup failed");
             ctx->have_tma = true;
         }
@@ -634,6 +634,7 @@ int32_t kvp_register_packet(kvp_ctx *ctx, const void *k, const void *v, int32_t 
     if (!ctx) return KVP_ERR_INVALID;
     if (!packet_id || n_tokens <= 0) return fail(ctx, KVP_ERR_INVALID, "register_packet: bad arguments");
     if (!ctx->host_only && (!k || !v)) return fail(ctx, KVP_ERR_INVALID, "register_packet: null K/V");
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(ctx, KVP_ERR_INVALID, "register_packet: K/V must be 16-byte aligned");
     if ((int)ctx->packets.size() >= ctx->cfg.max_packets) return fail(ctx, KVP_ERR_CAPACITY, "max_packets reached");
     if (ctx->pool_rows_used + n_tokens > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
     const int32_t rc = store_segment(ctx, k, v, n_tokens, (cudaStream_t)stream);
@@ -748,6 +749,8 @@ int32_t kvp_register_adapter(kvp_ctx *ctx, const void *hk, const void *hv, int32
     if (!adapter_id || n_header < 0 || n_trailer < 0) return fail(ctx, KVP_ERR_INVALID, "register_adapter: bad arguments");
     if (!ctx->host_only && ((n_header > 0 && (!hk || !hv)) || (n_trailer > 0 && (!tk || !tv))))
         return fail(ctx, KVP_ERR_INVALID, "register_adapter: null K/V");
+    if (((n_header > 0 ? ((uintptr_t)hk | (uintptr_t)hv) : 0) | (n_trailer > 0 ? ((uintptr_t)tk | (uintptr_t)tv) : 0)) & 15)
+        return fail(ctx, KVP_ERR_INVALID, "register_adapter: K/V must be 16-byte aligned");
     if ((int)ctx->adapter_h.size() >= ctx->cfg.max_adapters) return fail(ctx, KVP_ERR_CAPACITY, "max_adapters reached");
     if (ctx->pool_rows_used + n_header + n_trailer > ctx->shape.pool_rows) return fail(ctx, KVP_ERR_CAPACITY, "pool full");
     int32_t rc = store_segment(ctx, hk, hv, n_header, (cudaStream_t)stream);
@@ -1041,7 +1044,15 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "query_prefill: unknown assembly %d", assembly_id);
     if (!q || !k_new || !v_new || !out || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
         return fail(ctx, KVP_ERR_INVALID, "query_prefill: bad arguments");
-    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE | KVP_CONTINUE)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE | KVP_CONTINUE | KVP_PRECISE_QK)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    {
+        // every kernel reads whole elements; the tcgen05 path moves q and out 16 bytes at a time
+        const uintptr_t all = (uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)out;
+        if ((all & (uintptr_t)(ctx->shape.elem_bytes - 1)) || ((uintptr_t)lse & 3))
+            return fail(ctx, KVP_ERR_INVALID, "query_prefill: q / k_new / v_new / out / lse not aligned to their element size");
+        if (ctx->have_tma && !(flags & KVP_FORCE_SIMPLE) && ((((uintptr_t)q | (uintptr_t)out) & 15) != 0))
+            return fail(ctx, KVP_ERR_INVALID, "query_prefill: q and out must be 16-byte aligned on the tcgen05 path (KVP_FORCE_SIMPLE takes any element-aligned pointer)");
+    }
     if (q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_CAPACITY, "query_prefill: q_len > max_query_tokens");
     kvp_assembly_host &as = ctx->slots[slot];
     const kvp_shape &sh = ctx->shape;
@@ -1062,7 +1073,8 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
     // plain prefill on the two-stream kernel: it reads the query block's K/V from k_new / v_new and appends them itself
     kvp_attn2_args a;
     a.tail_direct = 0;
-    if (fast && ctx->kernel_variant == 0 && ctx->fused_append && !rope_query && q_pos0 == 0 &&
+    a.precise = (flags & KVP_PRECISE_QK) ? 1 : 0;
+    if (fast && ctx->fused_append && !rope_query && q_pos0 == 0 &&
         (((uintptr_t)k_new | (uintptr_t)v_new) & 15) == 0 &&
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_knew, k_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch) &&
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_vnew, v_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch))
@@ -1087,7 +1099,7 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
         KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
         ++launches;
         ctx->last_kind = 0;
-    } else if (ctx->kernel_variant == 0) {
+    } else {
         const int li = as.item_stride ? layer : 0;
         if (as.sched.empty()) as.sched.resize(as.item_stride ? ctx->cfg.n_layers : 1);
         const bool same_lens = q_lens ? (as.sched[li].q_lens.size() == (size_t)as.batch &&
@@ -1129,44 +1141,6 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
         ctas = ss.ctas;
         splits = ss.slots;
         ctx->last_kind = 1;
-    } else {
-        if (q_pos0 > 0 || as.item_stride) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: the single-tile kernel variant has no KVP_CONTINUE and no compressed packets");
-        const int n_mtiles = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
-        const int units = as.batch * sh.n_kv_heads * n_mtiles;
-        int min_tiles = INT32_MAX;
-        for (const kvp_item &it : as.items) min_tiles = std::min(min_tiles, it.tile_end - it.tile_begin + 1);
-        const int target = ctx->split_target_ctas > 0 ? ctx->split_target_ctas : 4 * ctx->sm_count;
-        if (units < target) {
-            splits = (target + units - 1) / units;
-            splits = std::min(splits, std::max(1, min_tiles / 4));
-            splits = std::min(splits, KVP_MAX_SPLIT_UNITS / units);
-            splits = std::max(splits, 1);
-        }
-        if (ctx->force_splits > 0) splits = std::min(ctx->force_splits, std::max(1, KVP_MAX_SPLIT_UNITS / units));
-        kvp_attn_sm100_args a;
-        a.plan = plan;
-        a.batch = as.batch;
-        a.q_len = q_len;
-        a.layer = layer;
-        a.n_splits = splits;
-        a.n_mtiles = n_mtiles;
-        a.q = q_used;
-        a.out = out;
-        a.lse = lse;
-        a.partial_o = ctx->partial_o;
-        a.partial_ml = ctx->partial_ml;
-        a.status = ctx->status_dev;
-        KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
-        KVP_CUDA(ctx, kvp_launch_attn_sm100_single(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot],
-                                            ctx->tm_ws_v[slot], &ctas, st));
-        KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
-        ++launches;
-        if (splits > 1) {
-            KVP_CUDA(ctx, kvp_launch_merge(sh, as.batch, q_len, splits, n_mtiles, ctx->partial_o, ctx->partial_ml, out,
-                                           lse, st));
-            ++launches;
-        }
-        ctx->last_kind = 1;
     }
     ctx->last_ctas = ctas;
     ctx->last_splits = splits;
@@ -1191,7 +1165,6 @@ int32_t kvp_query_prefill_ragged(kvp_ctx *ctx, int32_t assembly_id, int32_t laye
     for (int b = 0; b < ctx->slots[slot].batch; ++b)
         if (q_lens[b] < 1 || q_lens[b] > q_len_max)
             return fail(ctx, KVP_ERR_INVALID, "query_prefill_ragged: q_lens[%d] = %d outside [1, %d]", b, q_lens[b], q_len_max);
-    if (ctx->kernel_variant != 0) return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill_ragged: two-stream kernel only");
     return query_prefill_impl(ctx, assembly_id, layer, q, k_new, v_new, q_len_max, q_lens, 0, out, lse, stream);
 }
 
@@ -1204,7 +1177,7 @@ int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "segment_mass: unknown assembly %d", assembly_id);
     if (!q || !lse || !mass || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
         return fail(ctx, KVP_ERR_INVALID, "segment_mass: bad arguments");
-    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_CONTINUE | KVP_FORCE_SIMPLE)) return fail(ctx, KVP_ERR_INVALID, "segment_mass: unknown flags");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_CONTINUE | KVP_FORCE_SIMPLE | KVP_PRECISE_QK)) return fail(ctx, KVP_ERR_INVALID, "segment_mass: unknown flags");
     const kvp_assembly_host &as = ctx->slots[slot];
     if (ctx->shape.group > 8) return fail(ctx, KVP_ERR_UNSUPPORTED, "segment_mass: more than 8 q heads per kv head");
     if ((int)as.appended.size() != ctx->cfg.n_layers || as.appended[layer] < q_len)
@@ -1289,10 +1262,6 @@ int32_t kvp_tune(kvp_ctx *ctx, int32_t key, int32_t value)
         for (kvp_assembly_host &as : ctx->slots) as.sched.clear();       // work lists are rebuilt on next use
     }
     else if (key == KVP_TUNE_FUSED_APPEND) ctx->fused_append = value != 0;
-    else if (key == KVP_TUNE_KERNEL_VARIANT) {
-        if (value != 0 && value != 1) return fail(ctx, KVP_ERR_INVALID, "tune: kernel variant %d", value);
-        ctx->kernel_variant = value;
-    }
     else if (key == KVP_TUNE_TIME_KERNELS) {
         ctx->time_kernels = std::max(0, value);
         ctx->tev_n[0] = ctx->tev_n[1] = 0;

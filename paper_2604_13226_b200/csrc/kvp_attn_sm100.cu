@@ -70,6 +70,9 @@ struct Params {
     // tail_direct: the query block's tiles come from k_new / v_new ([batch][q_len][Hkv][d], through their own
     // tensor maps) and the kernel copies those rows into the workspace rows (the append) itself
     int tail_direct;
+    // precise: the counter-rotated query is kept as value + rounding remainder (two bf16 tiles per stream, one
+    // epoch buffer instead of two) and Q K^T of a rotated tile takes both
+    int precise;
     const uint4 *k_new, *v_new;
     uint4 *ws_k, *ws_v;
     long long ws_rows;
@@ -352,7 +355,9 @@ __device__ __forceinline__ int load_seq(int mode, int n, int r, int kv)
 // t >> 3, + 16, + 32, ...  The raw rows go to their place in the buffer by asynchronous copies, all in flight
 // together (one memory round trip for the tile, eight threads per 128-byte line); the thread then rotates
 // its own chunks in place.
-__device__ __forceinline__ void produce_q_tile(const Params &p, char *qbuf, int t, const __nv_bfloat16 *q_b, int hk,
+// With `qrem` (precise mode) the remainders r - bf16(r) of the rotated values go, as bf16, to the same places of
+// a second tile: q' = hi + rem to about 2^-17, so that the rounding of the re-based operand leaves the scores.
+__device__ __forceinline__ void produce_q_tile(const Params &p, char *qbuf, char *qrem, int t, const __nv_bfloat16 *q_b, int hk,
                                                int row_base, int n_rows, int rope)
 {
     const int c = t & 7, r0 = t >> 3;
@@ -388,14 +393,22 @@ __device__ __forceinline__ void produce_q_tile(const Params &p, char *qbuf, int 
         uint4 qa = *reinterpret_cast<uint4 *>(lo), qb = *reinterpret_cast<uint4 *>(lo + kHalfBytes);
         uint32_t *a = reinterpret_cast<uint32_t *>(&qa);
         uint32_t *b = reinterpret_cast<uint32_t *>(&qb);
+        uint4 ra, rb;                                            // remainders (precise mode)
+        uint32_t *ar = reinterpret_cast<uint32_t *>(&ra);
+        uint32_t *br = reinterpret_cast<uint32_t *>(&rb);
+        // word = bf16 pair of (x, y); rem = bf16 pair of what the rounding of the word dropped
+        auto put = [&](uint32_t &word, uint32_t &rem, float x, float y) {
+            word = pack_bf16(x, y);
+            rem = pack_bf16(x - lo_f(word), y - hi_f(word));
+        };
         if (p.pairing == 0) {
             // pairs (i, i + 64): word j of chunk c holds elements 8c+2j, 8c+2j+1; partners in chunk c+8
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const float4 w = w4[j];                          // cos, sin of pair 8c+2j; cos, sin of pair 8c+2j+1
                 const float a0 = lo_f(a[j]), a1 = hi_f(a[j]), b0 = lo_f(b[j]), b1 = hi_f(b[j]);
-                a[j] = pack_bf16(a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
-                b[j] = pack_bf16(b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
+                put(a[j], ar[j], a0 * w.x + b0 * w.y, a1 * w.z + b1 * w.w);     // R(-Delta): cos same, sin negated
+                put(b[j], br[j], b0 * w.x - a0 * w.y, b1 * w.z - a1 * w.w);
             }
         } else {
             // pairs (2i, 2i+1): one word each; chunk c holds pairs 4c..4c+3 (w4[0], w4[1]), chunk c+8 w4[2], w4[3]
@@ -403,16 +416,21 @@ __device__ __forceinline__ void produce_q_tile(const Params &p, char *qbuf, int 
             for (int j = 0; j < 4; j += 2) {
                 float4 w = w4[j >> 1];
                 float x0 = lo_f(a[j]), y0 = hi_f(a[j]), x1 = lo_f(a[j + 1]), y1 = hi_f(a[j + 1]);
-                a[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
-                a[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+                put(a[j], ar[j], x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                put(a[j + 1], ar[j + 1], x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
                 w = w4[2 + (j >> 1)];
                 x0 = lo_f(b[j]); y0 = hi_f(b[j]); x1 = lo_f(b[j + 1]); y1 = hi_f(b[j + 1]);
-                b[j] = pack_bf16(x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
-                b[j + 1] = pack_bf16(x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
+                put(b[j], br[j], x0 * w.x + y0 * w.y, y0 * w.x - x0 * w.y);
+                put(b[j + 1], br[j + 1], x1 * w.z + y1 * w.w, y1 * w.z - x1 * w.w);
             }
         }
         *reinterpret_cast<uint4 *>(lo) = qa;
         *reinterpret_cast<uint4 *>(lo + kHalfBytes) = qb;
+        if (qrem != nullptr) {
+            char *rl = qrem + (lo - qbuf);
+            *reinterpret_cast<uint4 *>(rl) = ra;
+            *reinterpret_cast<uint4 *>(rl + kHalfBytes) = rb;
+        }
     }
 }
 
@@ -687,13 +705,18 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
         const int max_steps = max(w.steps0, w.steps1);
         int prev0 = 0, prev1 = 0;
         auto produce = [&](int s, int rope, uint32_t &nEp) {
-            const int buf = nEp & 1;
-            if (nEp >= 2) {                                 // the epoch before last used this buffer
-                ok = mbar_wait(c.bar(kQFree + 2 * s + buf), ((nEp >> 1) - 1) & 1, c.abort_flag, p.status, 40 + s);
+            // two buffers per stream taken in turn; in precise mode one (value, remainder) pair, rewritten once
+            // the last Q K^T of the epoch before has run
+            const int buf = p.precise ? 0 : (nEp & 1);
+            const uint32_t back = p.precise ? 1u : 2u;      // the epoch that used this buffer last
+            if (nEp >= back) {
+                const uint32_t par = p.precise ? (nEp - 1) & 1 : ((nEp >> 1) - 1) & 1;
+                ok = mbar_wait(c.bar(kQFree + 2 * s + buf), par, c.abort_flag, p.status, 40 + s);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
             }
-            produce_q_tile(p, c.smem + kOffQ + (2 * s + buf) * kTileBytes, t, p.q + (long long)w.b * p.q_len * p.n_q * 128,
+            char *qb = c.smem + kOffQ + (2 * s + buf) * kTileBytes;
+            produce_q_tile(p, qb, p.precise ? qb + kTileBytes : nullptr, t, p.q + (long long)w.b * p.q_len * p.n_q * 128,
                            w.hk, w.row_base + (w.mode == 0 ? s * KVP_TILE_ROWS : 0), n_rows, rope);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(c.bar(kQFull + 2 * s + buf));
@@ -819,8 +842,8 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
         }
         const Tile tl = ms.cur;
         if (k == 0 || tl.rope != ms.prev_rope) {                  // first tile of a document: its own Q buffer
-            ms.qbuf = ms.nEpoch & 1;
-            ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
+            ms.qbuf = p.precise ? 0 : (ms.nEpoch & 1);
+            ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (p.precise ? ms.nEpoch : ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
             ++ms.nEpoch;
         }
         const int r = wq.mode ? 2 * k + s : k;
@@ -841,6 +864,15 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
             constexpr uint32_t kHalf16 = kHalfBytes >> 4;
             const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
             mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+        }
+        if (p.precise && tl.rope != 0) {                         // + (rounding remainder of the rotated Q) K^T
+            constexpr uint32_t kRem16 = kTileBytes >> 4;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                constexpr uint32_t kHalf16 = kHalfBytes >> 4;
+                const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
+                mma_ss<1>(d, desc64(q_lo + kRem16 + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+            }
         }
         tc_commit(c.bar(kSFull + s));
         if (!shared_stage || s == 1) tc_commit(c.bar(kKvEmpty + stage));
@@ -899,8 +931,8 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 }
                 if (k < n) {
                     if (newq) {
-                        ms.qbuf = ms.nEpoch & 1;
-                        if (ok) ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
+                        ms.qbuf = p.precise ? 0 : (ms.nEpoch & 1);
+                        if (ok) ok = mbar_wait(c.bar(kQFull + 2 * s + ms.qbuf), (p.precise ? ms.nEpoch : ms.nEpoch >> 1) & 1, c.abort_flag, p.status, 20 + s);
                         ++ms.nEpoch;
                     }
                 }
@@ -940,6 +972,15 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                         constexpr uint32_t kHalf16 = kHalfBytes >> 4;
                         const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
                         mma_ss<1>(d, desc64(q_lo + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+                    }
+                    if (p.precise && rope != 0) {                // + (rounding remainder of the rotated Q) K^T
+                        constexpr uint32_t kRem16 = kTileBytes >> 4;
+#pragma unroll 1
+                        for (int kk = 0; kk < 8; ++kk) {
+                            constexpr uint32_t kHalf16 = kHalfBytes >> 4;
+                            const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
+                            mma_ss<1>(d, desc64(q_lo + kRem16 + off, kDescHi), desc64(k_lo + off, kDescHi), idesc);
+                        }
                     }
                     tc_commit(c.bar(kSFull + s));
                     if (s == 1) tc_commit(c.bar(kKvEmpty + stK));
@@ -1185,6 +1226,7 @@ cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, 
     p.partial_ml = a.partial_ml;
     p.status = a.status;
     p.tail_direct = a.tail_direct;
+    p.precise = a.precise;
     p.k_new = (const uint4 *)a.k_new;
     p.v_new = (const uint4 *)a.v_new;
     p.ws_k = (uint4 *)a.ws_k;

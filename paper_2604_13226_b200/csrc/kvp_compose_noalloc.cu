@@ -14,6 +14,7 @@
 // or different host threads) race on the array; callers must serialise them.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <stdint.h>
 #include <stdio.h>
 
 #include <mutex>
@@ -163,6 +164,8 @@ extern "C" int32_t kvp_compose_noalloc(const void *pool_k, const void *pool_v, i
     if (err && err_cap > 0) err[0] = 0;
     if (!pool_k || !pool_v || !cache_k || !cache_v || !src_row0 || !seg_len || !delta)
         return report(err, err_cap, KVP_ERR_INVALID, "compose_noalloc: null pointer");
+    if (((uintptr_t)pool_k | (uintptr_t)pool_v | (uintptr_t)cache_k | (uintptr_t)cache_v) & 15)
+        return report(err, err_cap, KVP_ERR_INVALID, "compose_noalloc: pool and cache pointers must be 16-byte aligned");
     if (n_segments <= 0) return report(err, err_cap, KVP_ERR_INVALID, "compose_noalloc: n_segments must be positive");
     if (n_segments > kMaxSeg) {
         char msg[160];
@@ -181,6 +184,8 @@ extern "C" int32_t kvp_compose_noalloc(const void *pool_k, const void *pool_v, i
     for (int s = 0; s < n_segments; ++s) {
         if (seg_len[s] <= 0 || src_row0[s] < 0 || (int64_t)src_row0[s] + seg_len[s] > pool_rows)
             return report(err, err_cap, KVP_ERR_INVALID, "compose_noalloc: segment outside the pool");
+        if (dst + seg_len[s] > cache_rows || dst + seg_len[s] > (int64_t)INT32_MAX)     // before dst is narrowed below
+            return report(err, err_cap, KVP_ERR_CAPACITY, "compose_noalloc: segments do not fit in cache_rows");
         sp.src_row0[s] = src_row0[s];
         sp.len[s] = seg_len[s];
         sp.dst_row0[s] = (int32_t)dst;
@@ -188,7 +193,6 @@ extern "C" int32_t kvp_compose_noalloc(const void *pool_k, const void *pool_v, i
         dst += seg_len[s];
         if (seg_len[s] > max_len) max_len = seg_len[s];
     }
-    if (dst > cache_rows) return report(err, err_cap, KVP_ERR_CAPACITY, "compose_noalloc: segments do not fit in cache_rows");
 
     Scratch *sc = nullptr;
     cudaError_t e = scratch_on_current_device(&sc);

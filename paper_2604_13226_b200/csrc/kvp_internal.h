@@ -13,7 +13,7 @@
 #define KVP_TILE_KEYS 128      // keys per attention tile (one TMA box of K or V rows)
 #define KVP_TILE_ROWS 128      // packed query rows per CTA tile (MMA M)
 #define KVP_CHUNK_ROWS 32      // rows per gather work item
-#define KVP_MAX_SPLIT_UNITS 2048
+#define KVP_MAX_SPLIT_UNITS 2048   // partial slots (128 query rows each) in the workspace
 
 // ---- device-visible plan records (written by the host planner, uploaded once per assembly) -----
 
@@ -152,7 +152,6 @@ struct kvp_ctx {
     std::vector<cudaEvent_t> sched_event;
     uint64_t sched_off_works = 0, sched_off_merges = 0, sched_bytes = 0;
     int32_t sched_max_works = 0, sched_max_merges = 0;
-    int32_t kernel_variant = 0;            // 0: two-stream kernel, 1: single-tile kernel
     int32_t fused_append = 1;              // plain prefill: the attention kernel reads k_new / v_new itself and appends them
     void *encode_tiled = nullptr;          // cuTensorMapEncodeTiled
     float *partial_o = nullptr;            // [units][128][head_dim]
@@ -205,24 +204,6 @@ cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan
                                    const char *ws_k, const char *ws_v, void *out, float *lse, int32_t *ctas,
                                    cudaStream_t st);
 
-struct kvp_attn_sm100_args {
-    kvp_plan_dev plan;
-    int32_t batch, q_len, layer, n_splits, n_mtiles;
-    const void *q;
-    void *out;
-    float *lse;
-    float *partial_o;
-    float2 *partial_ml;
-    int32_t *status;
-};
-cudaError_t kvp_launch_merge(const kvp_shape &sh, int32_t batch, int32_t q_len, int32_t n_splits, int32_t n_mtiles,
-                             const float *partial_o, const float2 *partial_ml, void *out, float *lse,
-                             cudaStream_t st);
-cudaError_t kvp_attn_sm100_single_prepare(void);
-cudaError_t kvp_launch_attn_sm100_single(const kvp_shape &sh, const kvp_attn_sm100_args &a, const CUtensorMap &tm_pool_k,
-                                         const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
-                                         const CUtensorMap &tm_ws_v, int32_t *ctas, cudaStream_t st);
-
 struct kvp_attn2_args {
     kvp_plan_dev plan;
     int32_t q_len, q_pos0, layer, n_ctas;
@@ -237,6 +218,7 @@ struct kvp_attn2_args {
     // tail_direct: the query block's K/V tiles are loaded from k_new / v_new ([batch][q_len][Hkv][d]) through
     // tm_knew / tm_vnew and the kernel copies those rows into the workspace rows itself
     int32_t tail_direct;
+    int32_t precise;               // KVP_PRECISE_QK
     const void *k_new, *v_new;
     char *ws_k, *ws_v;
     CUtensorMap tm_knew, tm_vnew;

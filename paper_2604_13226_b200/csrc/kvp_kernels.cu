@@ -449,40 +449,6 @@ segment_mass_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T
         out[(int64_t)(w / (n_cols - n_seg - 1)) * n_cols + n_seg + 1 + w % (n_cols - n_seg - 1)] = 0.f;
 }
 
-// ---- split-KV merge -----------------------------------------------------------------------------
-// Partials hold, per (unit, row): un-normalised O (fp32), the running max m of the raw scores and
-// the sum l of exp2((s - m) * c).  One block per (b, hk, m-tile, 16-row group), one thread per column.
-template <typename T>
-__global__ void merge_kernel(int q_len, int n_q, int n_kv, int group, int d, int n_splits, int n_mtiles, float scale,
-                             const float *__restrict__ part_o, const float2 *__restrict__ part_ml,
-                             T *__restrict__ out, float *__restrict__ lse)
-{
-    const int u = blockIdx.x;                       // (b*Hkv + hk)*n_mtiles + mt
-    const int mt = u % n_mtiles;
-    const int hk = (u / n_mtiles) % n_kv;
-    const int b = u / (n_mtiles * n_kv);
-    const float c2 = scale * 1.4426950408889634f;
-    const int c = threadIdx.x;
-    for (int rr = 0; rr < 16; ++rr) {
-        const int row = blockIdx.y * 16 + rr;
-        const int r = mt * KVP_TILE_ROWS + row;
-        if (r >= group * q_len) break;
-        float M = -INFINITY;
-        for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[((int64_t)u * n_splits + s) * KVP_TILE_ROWS + row].x);
-        float L = 0.f, o = 0.f;
-        for (int s = 0; s < n_splits; ++s) {
-            const int64_t base = ((int64_t)u * n_splits + s) * KVP_TILE_ROWS + row;
-            const float2 ml = part_ml[base];
-            const float w = exp2f((ml.x - M) * c2);
-            L += w * ml.y;
-            if (c < d) o += w * part_o[base * d + c];
-        }
-        const int i = r / group, h = hk * group + r % group;
-        if (c < d) out[(((int64_t)b * q_len + i) * n_q + h) * d + c] = Elem<T>::from_f32(o / L);
-        if (c == 0 && lse != nullptr) lse[((int64_t)b * n_q + h) * q_len + i] = M * scale + logf(L);
-    }
-}
-
 }  // namespace
 
 // ---- launchers ------------------------------------------------------------------------------------
@@ -588,19 +554,5 @@ cudaError_t kvp_launch_attn_simple(const kvp_shape &sh, const kvp_plan_dev &plan
         if (sh.head_dim == 128) KVP_SIMPLE(float, 128); else KVP_SIMPLE(float, 64);
     }
 #undef KVP_SIMPLE
-    return cudaGetLastError();
-}
-
-cudaError_t kvp_launch_merge(const kvp_shape &sh, int32_t batch, int32_t q_len, int32_t n_splits, int32_t n_mtiles,
-                             const float *partial_o, const float2 *partial_ml, void *out, float *lse, cudaStream_t st)
-{
-    const dim3 grid(batch * sh.n_kv_heads * n_mtiles, KVP_TILE_ROWS / 16);
-    if (sh.dtype == KVP_DTYPE_BF16)
-        merge_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>(q_len, sh.n_q_heads, sh.n_kv_heads, sh.group, sh.head_dim,
-                                                         n_splits, n_mtiles, sh.scale, partial_o, partial_ml,
-                                                         (__nv_bfloat16 *)out, lse);
-    else
-        merge_kernel<float><<<grid, 128, 0, st>>>(q_len, sh.n_q_heads, sh.n_kv_heads, sh.group, sh.head_dim, n_splits,
-                                                 n_mtiles, sh.scale, partial_o, partial_ml, (float *)out, lse);
     return cudaGetLastError();
 }

@@ -72,10 +72,6 @@ def test_compressed_unsupported_paths_and_validation():
     with pytest.raises(kvp.KvpError) as e:
         sess.ctx.export_cache(aid, 0, 0, plen[0], 0)
     assert e.value.code == 5
-    sess.ctx.tune(kvp.TUNE_KERNEL_VARIANT, 1)
-    with pytest.raises(kvp.KvpError) as e:
-        sess.prefill(0)
-    assert e.value.code == 5
     with pytest.raises(kvp.KvpError) as e:
         sess.ctx.assemble(wl.items, kvp.REBASE | kvp.MATERIALIZE)
     assert e.value.code == 5

@@ -108,6 +108,39 @@ def test_argument_errors_are_status_codes():
     ctx.close()
 
 
+def test_misaligned_pointers_are_refused_on_the_host():
+    # 16-byte vector accesses need 16-byte aligned pointers; the check comes before any CUDA call, so it can be
+    # exercised without a device (the addresses are never dereferenced)
+    wl = ragged_workload()
+    ctx = host_ctx(wl.shape, wl, max_slots=8)
+    for k, v in ((4096 + 8, 4096), (4096, 4096 + 2)):
+        with pytest.raises(kvp.KvpError) as e:
+            ctx.register_packet(k, v, 4, 0)
+        assert e.value.code == 1 and "aligned" in str(e.value)
+    with pytest.raises(kvp.KvpError) as e:
+        ctx.register_adapter(4096, 4096, 2, 0, 4096, 4096 + 4, 2, 0)
+    assert e.value.code == 1 and "aligned" in str(e.value)
+    ctx.close()
+    ok = 1 << 20
+    for bad in range(4):
+        ptrs = [ok, ok, ok, ok]
+        ptrs[bad] += 8
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.compose_noalloc(ptrs[0], ptrs[1], 64, 4, 128, "bf16", 0, 10000.0, [(0, 8, 0)], ptrs[2], ptrs[3], 128)
+        assert e.value.code == 1 and "aligned" in str(e.value)
+    # the running row count is checked before it is narrowed to 32 bits
+    big = [(0, 2 ** 31 - 8, 0), (0, 2 ** 31 - 8, 0)]
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.compose_noalloc(ok, ok, 2 ** 31 - 1, 1, 128, "bf16", 0, 10000.0, big, ok, ok, 2 ** 33)
+    assert e.value.code == 2
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.compose_noalloc(ok, ok, 64, 4, 128, "bf16", 0, 10000.0, [(0, 1, 0)] * 97, ok, ok, 128)
+    assert e.value.code == 2 and "96" in str(e.value)
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.compose_noalloc(ok, ok, 64, 4, 128, "bf16", 0, 10000.0, [(60, 10, 0)], ok, ok, 128)
+    assert e.value.code == 1
+
+
 def test_bad_configurations_rejected():
     for kw in (dict(n_q_heads=5, n_kv_heads=2), dict(head_dim=96), dict(n_layers=0)):
         args = dict(n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64)
