@@ -65,8 +65,8 @@ bool valid_cfg(const kvp_config *c)
 kvp_plan_layout plan_layout(const kvp_config *c)
 {
     kvp_plan_layout p;
-    // with compressed packets every layer has its own item records and tile list
-    const int64_t lists = c->max_compressed > 0 ? c->n_layers : 1;
+    // with compressed packets every (layer, kv head) has its own item records and tile list
+    const int64_t lists = c->max_compressed > 0 ? (int64_t)c->n_layers * c->n_kv_heads : 1;
     p.max_segs = 3 * c->max_slots;
     p.max_rope = p.max_segs + 1;
     p.max_items = (int32_t)(c->max_batch * lists);
@@ -228,11 +228,11 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     // that hold them reach the same key tiles at the same time and all but the first find them in L2.
     for (int row_base = 0; row_base < max_rows; row_base += 2 * KVP_TILE_ROWS)
         for (int b = 0; b < as.batch; ++b) {
-            const kvp_item &item = as.items[(as.item_stride ? layer * as.item_stride : 0) + b];
-            const int n_prefix = item.tile_end - item.tile_begin;
             const int n_rows = sh.group * (q_lens ? q_lens[b] : q_len);
             if (row_base >= n_rows) continue;
             for (int hk = 0; hk < sh.n_kv_heads; ++hk) {
+                const kvp_item &item = as.items[(as.item_stride ? (layer * sh.n_kv_heads + hk) * as.item_stride : 0) + b];
+                const int n_prefix = item.tile_end - item.tile_begin;
                 unit_t u;
                 u.q_len = q_lens ? q_lens[b] : 0;
                 u.b = b; u.hk = hk; u.row_base = row_base;
@@ -813,12 +813,9 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
         for (int32_t o = 0; o < n; o += KVP_CHUNK_ROWS)
             chunks.push_back({src + o, dst + o, std::min<int32_t>(KVP_CHUNK_ROWS, n - o), rope});
     };
-    // kept_row < 0: every plane holds all n rows; else the run belongs to a compressed packet whose
-    // per-plane counts are row kept_row of the assembly's table, and n is the largest of this layer's
-    auto add_tiles = [&](int16_t src, int32_t row0, int32_t n, int32_t rope, int32_t kept_row) {
+    auto add_tiles = [&](int16_t src, int32_t row0, int32_t n, int32_t rope) {
         for (int32_t o = 0; o < n; o += KVP_TILE_KEYS)
-            as.tiles.push_back({row0 + o, (int16_t)std::min<int32_t>(KVP_TILE_KEYS, n - o), src, rope,
-                                kept_row < 0 ? -1 : (kept_row << 16) | (o / KVP_TILE_KEYS)});
+            as.tiles.push_back({row0 + o, (int16_t)std::min<int32_t>(KVP_TILE_KEYS, n - o), src, rope, 0});
     };
     std::map<int32_t, int32_t> kept_row_of;    // compressed packet id -> row of the kept table
     std::vector<int32_t> kept_packets;
@@ -880,7 +877,7 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
                 kvp_seg &e = as.segs[s];
                 add_chunks(e.src_row0, it.cache_row0 + e.dst_pos0, e.len, e.rope);
             }
-            add_tiles(1, it.cache_row0, it.prefix_len, 0, -1);
+            add_tiles(1, it.cache_row0, it.prefix_len, 0);
             it.tail_row0 = it.cache_row0 + it.prefix_len;
             it.tile_end = (int32_t)as.tiles.size();
             ws_cursor += (int64_t)it.prefix_len + cfg.max_query_tokens;
@@ -904,26 +901,25 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
     }
     if ((int)kept_packets.size() > cfg.max_compressed)
         return fail(ctx, KVP_ERR_CAPACITY, "assemble: %zu compressed packets > max_compressed", kept_packets.size());
-    // tile lists: one for all layers, or - when a compressed packet keeps a different number of rows per
-    // layer - one per layer (documents are read in place; the staged adapter rows come first)
-    const int n_lists = kept_packets.empty() ? 1 : cfg.n_layers;
+    // tile lists: one for all planes, or - when a compressed packet keeps a different number of rows per
+    // (layer, kv head) - one per plane, so that a head walks exactly the tiles it holds (documents are read
+    // in place; the staged adapter rows come first)
+    const int n_lists = kept_packets.empty() ? 1 : cfg.n_layers * cfg.n_kv_heads;
     as.item_stride = kept_packets.empty() ? 0 : batch;
     for (int l = 0; l < n_lists; ++l)
         for (int b = 0; b < batch; ++b) {
             kvp_item it = builds[b].it;
             if (!mat) {
                 it.tile_begin = (int32_t)as.tiles.size();
-                add_tiles(1, builds[b].stage0, builds[b].staged, 0, -1);
+                add_tiles(1, builds[b].stage0, builds[b].staged, 0);
                 for (int s = it.seg_begin; s < it.seg_end; ++s) {
                     const kvp_seg &e = as.segs[s];
                     if (e.pad[1] != 1) continue;
                     if (e.pad[2] < 0) {
-                        add_tiles(0, e.src_row0, e.len, e.rope, -1);
+                        add_tiles(0, e.src_row0, e.len, e.rope);
                     } else {
                         const std::vector<int32_t> &kept = ctx->packets[kept_packets[e.pad[2]]].kept;
-                        int32_t n_l = 0;
-                        for (int h = 0; h < cfg.n_kv_heads; ++h) n_l = std::max(n_l, kept[l * cfg.n_kv_heads + h]);
-                        add_tiles(0, e.src_row0, n_l, e.rope, e.pad[2]);
+                        add_tiles(0, e.src_row0, kept[l], e.rope);              // l = layer * n_kv_heads + kv head
                     }
                 }
                 it.tile_end = (int32_t)as.tiles.size();

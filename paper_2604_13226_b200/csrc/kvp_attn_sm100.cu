@@ -295,7 +295,7 @@ __device__ __forceinline__ Work load_work(const Params &p, int wi)
     w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w & 0xff;
     w.q_len = (a.w >> 8) ? (a.w >> 8) : p.q_len;
     w.lo = c.x; w.n = c.y; w.slot0 = c.z; w.slot1 = c.w;
-    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + p.layer * p.plan.item_stride + w.b);
+    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + (p.layer * p.n_kv + w.hk) * p.plan.item_stride + w.b);
     const int4 ia = __ldg(i4), ib = __ldg(i4 + 1);          // prefix_len, tile_begin, tile_end, seg_begin | seg_end, tail_row0, ..
     w.tile_begin = ia.y;
     w.tail_row0 = ib.y;
@@ -329,10 +329,6 @@ __device__ __forceinline__ Tile get_tile(const Params &p, const Work &w, int j)
         t.src = g.y >> 16;
         t.rope = g.z;
         t.qoff = -1;
-        if (g.w >= 0) {        // compressed packet: this (layer, kv head) keeps fewer rows, possibly none of this tile
-            const int kept = __ldg(p.plan.kept + (g.w >> 16) * p.plan.n_planes + w.plane);
-            t.n_keys = max(0, min(t.n_keys, kept - (g.w & 0xFFFF) * KVP_TILE_KEYS));
-        }
     }
     return t;
 }
@@ -601,8 +597,10 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Cta &c, cons
                 tmem_st16(s_addr + ch * 16, pk);
                 l += ls;
             };
+            // a short tile (the end of a document, staged adapter rows) needs P only for the columns P V will read
+            const int n_ch = full ? 4 : max(1, (tl.n_keys + 31) >> 5);
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < n_ch; ++ch) {
                 tmem_ld32(s_addr + ch * 32, va);
                 tc_wait_ld();
                 landed32(va);
@@ -853,7 +851,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
         ok = __all_sync(0xffffffffu, ok);                         // the lanes stay together
         if (!ok) return;
         tc_fence_after();
-        const uint32_t n16 = max(16u, (uint32_t)(tl.n_keys + 15) & ~15u);      // a tile may be empty for this head
+        const uint32_t n16 = max(16u, (uint32_t)(tl.n_keys + 15) & ~15u);
         const uint32_t idesc = instr_desc(n16, 0);
         const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
         const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stage * kTileBytes, 16);
@@ -961,7 +959,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                 }
                 if (k < n) {
                     // ---- S_s = Q_s K^T of step k ----------------------------------------------------
-                    const uint32_t n16 = max(16u, (uint32_t)(nk + 15) & ~15u);         // a tile may be empty for this head
+                    const uint32_t n16 = max(16u, (uint32_t)(nk + 15) & ~15u);   
                     const uint32_t idesc = instr_desc(n16, 0);
                     const uint32_t q_lo = desc_lo(c.smem_base + kOffQ + (2 * s + ms.qbuf) * kTileBytes, 16);
                     const uint32_t k_lo = desc_lo(c.smem_base + kOffRing + stK * kTileBytes, 16);

@@ -22,8 +22,7 @@ struct kvp_tile {              // one run of <= 128 consecutive key rows sharing
     int16_t n_keys;            // 1..128
     int16_t src;               // 0 pool, 1 workspace
     int32_t rope;              // rope-table index of the offset still to be applied to these keys (0 = none)
-    int32_t clip;              // -1, or (row of the kept-count table << 16) | tile number inside the packet:
-                               // plane (layer, kv head) then holds only kept - 128 * tile number of these keys
+    int32_t pad;
 };
 
 struct kvp_chunk {             // gather work item: <= 32 rows copied pool -> workspace, keys rotated
@@ -88,7 +87,7 @@ struct kvp_plan_dev {
     const kvp_seg *segs;
     const float2 *rope;        // [n_rope][head_dim/2] (cos, sin) of delta * theta_i
     const int32_t *kept;       // [compressed packets of the assembly][n_layers * n_kv_heads] kept rows per plane
-    int32_t item_stride;       // 0: one item / tile list for all layers; batch: items[layer * batch + b]
+    int32_t item_stride;       // 0: one item / tile list for all planes; batch: items[(layer * n_kv_heads + kv head) * batch + b]
     int32_t n_planes;
 };
 
@@ -114,7 +113,7 @@ struct kvp_assembly_host {
     std::vector<kvp_seg> segs;
     std::vector<kvp_tile> tiles;
     int32_t n_chunks = 0, n_rope = 0;
-    int32_t item_stride = 0;               // batch when the assembly has per-layer tile lists (compressed packets)
+    int32_t item_stride = 0;               // batch when the assembly has a tile list per (layer, kv head) (compressed packets)
     int32_t last_q_len = 0;
     std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
     bool ragged = false;                   // a kvp_query_prefill_ragged call has appended a different number of rows per request

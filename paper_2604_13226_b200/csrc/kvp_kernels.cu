@@ -253,7 +253,7 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T 
     __shared__ float Ps[RB][KC];
 
     const int hk = blockIdx.y, b = blockIdx.z;
-    const kvp_item it = plan.items[layer * plan.item_stride + b];
+    const kvp_item it = plan.items[(layer * n_kv + hk) * plan.item_stride + b];
     const int n_rows = group * q_len;
     const int row = threadIdx.x / 8, sub = threadIdx.x % 8;
     const int r = blockIdx.x * RB + row;
@@ -290,10 +290,6 @@ attn_simple_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T 
             qoff = tt * KVP_TILE_KEYS;
         } else {
             tl = plan.tiles[it.tile_begin + tt - n_tail];
-            if (tl.clip >= 0) {      // compressed packet: rows kept by this (layer, kv head)
-                const int kept = plan.kept[(tl.clip >> 16) * plan.n_planes + plane];
-                tl.n_keys = (int16_t)max(0, min((int)tl.n_keys, kept - (tl.clip & 0xFFFF) * KVP_TILE_KEYS));
-            }
         }
         const int64_t prow = (tl.src == 0) ? (int64_t)plane * pool_rows : (int64_t)plane * ws_rows;
         const T *kb = reinterpret_cast<const T *>(tl.src == 0 ? pool_k : ws_k) + (prow + tl.row0) * D;
@@ -387,7 +383,7 @@ segment_mass_kernel(kvp_plan_dev plan, int q_len, int q_pos0, int layer, const T
     extern __shared__ float sm[];                            // [group][D] q rows, [8][group] partial sums, [group] lse
     float *qs = sm, *part = sm + group * D, *ls = part + 8 * group;
     const int b = blockIdx.x / q_len, i = blockIdx.x % q_len, hk = blockIdx.y;
-    const kvp_item it = plan.items[layer * plan.item_stride + b];
+    const kvp_item it = plan.items[(layer * n_kv + hk) * plan.item_stride + b];
     const int plane = layer * n_kv + hk;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int w = threadIdx.x; w < group * D; w += blockDim.x)
