@@ -446,6 +446,142 @@ def measure_host_packets_point(seed: int, iters: int, device: int, n_layers: int
 
 
 # ---------------------------------------------------------------------------------------------------
+# second scaling mode: prefix sharding (the packets of every request spread over the ranks)
+# ---------------------------------------------------------------------------------------------------
+
+def run_prefix_shard(args, rank: int, world: int, local_rank: int, peaks):
+    """`--shard prefix`: strong scaling of one long-context batch.  Rank r holds packets [r n/N, (r+1) n/N) of every
+    request (`kvp_assemble_at` re-bases them to their positions in the whole request), attends to them with
+    KVP_PARTIAL (the last rank also takes the query's own keys), the partial (O, m, l) buffers are all-gathered into
+    local memory over NCCL - the path's one exchange - and every rank merges them (`kvp_merge_partials`).  No kernel
+    is given a peer's memory."""
+    import torch
+    from paper_2604_13226_b200 import binding as kvp, inputs as gen
+    from paper_2604_13226_b200.session import Session
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device(f"cuda:{local_rank}")
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    name = args.workload if args.workload.startswith("config5") else "config5:64:16:1"
+    _, n, ql, b = name.split(":")
+    n, ql, b = int(n), int(ql), int(b)
+    if n % world:
+        raise SystemExit(f"--shard prefix: {n} packets per request do not divide over {world} ranks")
+    per_rank = n // world
+    whole = gen.spec_config5(n, ql, b, seed=args.seed)
+    spec = gen.spec_config5(per_rank, ql, b, seed=args.seed + 17 * rank)          # this rank's packets (its own draws)
+    doc = spec.packet_lens[0] + spec.n_header + spec.n_trailer
+    pos_base = [rank * per_rank * doc] * b
+    s = spec.shape
+    wl = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
+    sess = Session(wl, device=local_rank)
+    L = s.n_layers
+    # the query is the same on every rank: drawn from the whole request's seed
+    qkv = [gen.DeviceWorkload(whole, f"cuda:{local_rank}").query_device(l) for l in range(L)]
+    part_bytes = sess.ctx.partial_bytes(b, ql)
+    part = torch.empty(part_bytes, dtype=torch.uint8, device=dev)
+    gathered = torch.empty(part_bytes * world, dtype=torch.uint8, device=dev) if world > 1 else part
+    outs = [torch.empty_like(qkv[l][0]) for l in range(L)]
+    flags = kvp.PARTIAL | (0 if rank == world - 1 else kvp.SKIP_QUERY_BLOCK)
+
+    def layer(l, q, kn, vn, out):
+        sess.ctx.query_prefill(sess.assembly_id, l, q, kn, vn, ql, part, None, flags)
+        if world > 1:
+            dist.all_gather_into_tensor(gathered, part)                        # NCCL, into this GPU's own memory
+        sess.ctx.merge_partials(gathered, world, b, ql, out, None)
+
+    def step():
+        sess.assemble(pos_base=pos_base)
+        for l in range(L):
+            layer(l, *qkv[l], outs[l])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    launches_per_step = 1 + L * (sess.ctx.last_launch()["launches"] + 1)
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 1)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.1)
+    def timed(fn):
+        """K steps, each bracketed by a barrier + synchronize and timed with its own event pair; L2 is flushed
+        between them, outside the timed parts (a rank's share of the keys can be smaller than L2)."""
+        total = 0.0
+        for _ in range(args.steps):
+            flush_l2(torch, dev)
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            barrier()
+            total += e0.elapsed_time(e1)
+        return total
+
+    t0 = ClockSampler.now()
+    ms_total = timed(step)
+    clocks = sampler.window(t0, ClockSampler.now()) if rank == 0 else None
+    sampler.stop()
+    attn_ms = sess.ctx.kernel_times(0)
+    sess.ctx.tune(kvp.TUNE_TIME_KERNELS, 0)
+    assert sess.ctx.status_word() == 0
+    # end to end: the query chunk comes from pinned host memory and the output goes back, inside the timed region
+    hq = [tuple(t.cpu().pin_memory() for t in qkv[l]) for l in range(L)]
+    hout = [torch.empty_like(outs[l], device="cpu").pin_memory() for l in range(L)]
+    dq = tuple(torch.empty_like(t) for t in qkv[0])
+    dout = torch.empty_like(outs[0])
+
+    def step_e2e():
+        sess.assemble(pos_base=pos_base)
+        for l in range(L):
+            for dst, src in zip(dq, hq[l]):
+                dst.copy_(src, non_blocking=True)
+            layer(l, *dq, dout)
+            hout[l].copy_(dout, non_blocking=True)
+
+    for _ in range(3):
+        step_e2e()
+    ms_e2e = timed(step_e2e)
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, dev)
+    h2d = sum(t.numel() * t.element_size() for t in hq[0]) * L
+    d2h = hout[0].numel() * hout[0].element_size() * L
+    sess.close()
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        flops, bytes_ = algorithmic_work(spec)                                 # this rank's share of the keys
+        a_ms = statistics.mean(attn_ms) if attn_ms else None
+        roof = None
+        if a_ms:
+            ach = bytes_ / a_ms / 1e6
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                    "frac_nominal": ach / NOMINAL_GBS, "peak_nominal": NOMINAL_GBS, "traffic": None, "peak_source": peaks["source"],
+                    "kernel": "attn_sm100_kernel (one rank's keys)", "launches_timed": len(attn_ms), "avg_launch_ms": a_ms,
+                    "algorithmic_bytes_per_launch": bytes_, "algorithmic_flops_per_launch": flops}
+        cfg = workload_config(whole, False, bytes_)
+        cfg.update({"sharding": "prefix: the packets of every request split over the ranks; per layer one all-gather of "
+                                "(O, m, l) partials into local memory and a log-sum-exp merge",
+                    "packets_per_rank": per_rank, "exchange_bytes_per_rank_per_layer": part_bytes,
+                    "l2": "L2 flushed between steps, outside the timed parts (every step has its own event pair)"})
+        print(json.dumps({
+            "metric": "composed_cache_prefill_query_tokens_per_s", "value": b * ql / (ms_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
+            "e2e": {"value": b * ql / (ms_e2e / args.steps * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e / args.steps,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * args.steps, "roofline": roof, "clocks": clocks}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------------
 # main
 # ---------------------------------------------------------------------------------------------------
 
@@ -459,6 +595,9 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the extra roofline points and the CPU baseline")
     ap.add_argument("--materialize", action="store_true", help="materialise the composed prefix instead of reading in place")
+    ap.add_argument("--shard", default="requests", choices=["requests", "prefix"],
+                    help="requests: every rank its own batch (weak scaling, the default); prefix: the packets of one "
+                         "long-context batch (config5:<packets>:<q_len>:<batch>) split over the ranks (strong scaling)")
     ap.add_argument("--sweep", action="store_true",
                     help="time the attention kernel over the config-5 grid (packets x q_len x batch) and print one JSON line per point")
     args = ap.parse_args()
@@ -515,6 +654,10 @@ def main():
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
             "cpu_baseline": cb, "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0, "wall_s": dt}))
+        return
+
+    if args.shard == "prefix":
+        run_prefix_shard(args, rank, world, local_rank, peaks)
         return
 
     # ---- our arm ---------------------------------------------------------------------------------

@@ -56,7 +56,9 @@ enum {
     KVP_ROPE_QUERY = 1u,      /* q and k_new are raw: rotate them at positions prefix_len[b] + i        */
     KVP_FORCE_SIMPLE = 2u,    /* use the plain fp32 CUDA-core kernel (cross-check path, any dtype)      */
     KVP_CONTINUE = 4u,        /* the q_len tokens follow the rows this layer's earlier calls appended   */
-    KVP_PRECISE_QK = 8u       /* tcgen05 path: carry the re-based operand of q.k in two bf16 numbers    */
+    KVP_PRECISE_QK = 8u,      /* tcgen05 path: carry the re-based operand of q.k in two bf16 numbers    */
+    KVP_PARTIAL = 16u,        /* `out` receives un-normalised partial results (see kvp_merge_partials)  */
+    KVP_SKIP_QUERY_BLOCK = 32u /* with KVP_PARTIAL: leave the query's own keys to another rank           */
 };
 
 typedef struct kvp_ctx kvp_ctx;
@@ -190,6 +192,20 @@ KVP_API int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_of
                      void *stream, int32_t *prefix_len, int32_t *assembly_id);
 
 /*
+ * The same composition for one shard of a request whose packets are spread over several GPUs (the paper scales
+ * context by adding packets - the long-context settings of Section 4.3 - and a request's packets are independent
+ * units, Section 3.1, so a rank can hold any subset of them).  Request b's slots here are a contiguous part of
+ * its full slot list; pos_base[b] (host, [batch], >= 0) is the position at which that part starts in the full
+ * composed sequence, i.e. the total length of the slots before it, adapters included.  Every key is re-based to
+ * its position in the full sequence: Delta = pos_base[b] + offset within this part - cache position (Eq. 1).
+ * prefix_len[b] receives the number of tokens of this part.  Everything else as kvp_assemble.  On such an
+ * assembly kvp_query_prefill refuses KVP_ROPE_QUERY (the query's position is not prefix_len[b]).
+ */
+KVP_API int32_t kvp_assemble_at(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets,
+                        const int32_t *packet_ids, const int32_t *adapter_ids, const int32_t *pos_base,
+                        uint32_t flags, void *stream, int32_t *prefix_len, int32_t *assembly_id);
+
+/*
  * Query prefill of one layer over an assembly (Section 3.2 step 4; Fig. 2(d)): query token i of
  * request b attends to all prefix_len[b] composed tokens and to query tokens <= i, softmax in fp32,
  * q head h using kv head h / (Hq/Hkv).  k_new / v_new are appended to the request's cache at rows
@@ -219,6 +235,21 @@ KVP_API int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_of
 KVP_API int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q,
                           const void *k_new, const void *v_new, int32_t q_len, uint32_t flags,
                           void *out, float *lse, void *stream);
+
+/* Size in bytes of the buffer a KVP_PARTIAL prefill of `batch` requests x `q_len` tokens writes.  0 if invalid. */
+KVP_API uint64_t kvp_partial_bytes(kvp_ctx *ctx, int32_t batch, int32_t q_len);
+
+/*
+ * Combine the partial results of the ranks of a prefix-sharded request into the attention output: per query row
+ * M = max m_r, L = sum_r l_r 2^((m_r - M) c), O = sum_r O_r 2^((m_r - M) c) / L - softmax attention over the union
+ * of the ranks' keys (Section 3.2 step 4 over the whole composed sequence).
+ *   parts   device: n_parts buffers of kvp_partial_bytes(ctx, batch, q_len) bytes back to back (what an
+ *           all-gather of the ranks' buffers delivers), 16-byte aligned, all in this GPU's memory
+ *   out     device [batch][q_len][n_q_heads][head_dim], lse device float [batch][n_q_heads][q_len] or NULL
+ * Errors: INVALID, CAPACITY (batch / q_len beyond the context's maxima), STATE, UNSUPPORTED (not bf16 / 128), CUDA.
+ */
+KVP_API int32_t kvp_merge_partials(kvp_ctx *ctx, const void *parts, int32_t n_parts, int32_t batch, int32_t q_len,
+                           void *out, float *lse, void *stream);
 
 /*
  * The same for a batch whose requests bring query chunks of different lengths (a serving batch rarely has equal

@@ -18,7 +18,7 @@ STATUS_NAMES = {0: "KVP_OK", 1: "KVP_ERR_INVALID", 2: "KVP_ERR_CAPACITY", 3: "KV
                 4: "KVP_ERR_STATE", 5: "KVP_ERR_UNSUPPORTED", 6: "KVP_ERR_CUDA", 7: "KVP_ERR_TIMEOUT"}
 DTYPE_F32, DTYPE_BF16 = 0, 1
 REBASE, MATERIALIZE = 1, 2
-ROPE_QUERY, FORCE_SIMPLE, CONTINUE, PRECISE_QK = 1, 2, 4, 8
+ROPE_QUERY, FORCE_SIMPLE, CONTINUE, PRECISE_QK, PARTIAL, SKIP_QUERY_BLOCK = 1, 2, 4, 8, 16, 32
 TUNE_SPLIT_TARGET_CTAS, TUNE_FORCE_SPLITS, TUNE_TIME_KERNELS, TUNE_FUSED_APPEND = 1, 2, 3, 5
 
 
@@ -69,6 +69,9 @@ def lib() -> ctypes.CDLL:
         "kvp_evict_packet": (i32, [vp, i32]),
         "kvp_register_adapter": (i32, [vp, vp, vp, i32, i32, vp, vp, i32, i32, vp, pi32]),
         "kvp_assemble": (i32, [vp, i32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
+        "kvp_assemble_at": (i32, [vp, i32, pi32, pi32, pi32, pi32, u32, vp, pi32, pi32]),
+        "kvp_partial_bytes": (u64, [vp, i32, i32]),
+        "kvp_merge_partials": (i32, [vp, vp, i32, i32, i32, vp, vp, vp]),
         "kvp_query_prefill": (i32, [vp, i32, i32, vp, vp, vp, i32, u32, vp, vp, vp]),
         "kvp_query_prefill_ragged": (i32, [vp, i32, i32, vp, vp, vp, i32, pi32, vp, vp, vp]),
         "kvp_export_plan": (i32, [vp, i32, i32, pi32, pi32, pi32, pi32]),
@@ -93,7 +96,7 @@ def lib() -> ctypes.CDLL:
 
 EXPORTED = ["kvp_version", "kvp_token_bytes", "kvp_workspace_bytes", "kvp_create", "kvp_destroy",
             "kvp_register_packet", "kvp_register_packet_compressed", "kvp_register_packet_host", "kvp_evict_packet",
-            "kvp_register_adapter", "kvp_assemble", "kvp_query_prefill", "kvp_query_prefill_ragged",
+            "kvp_register_adapter", "kvp_assemble", "kvp_assemble_at", "kvp_partial_bytes", "kvp_merge_partials", "kvp_query_prefill", "kvp_query_prefill_ragged",
             "kvp_export_plan", "kvp_export_cache", "kvp_export_schedule", "kvp_segment_mass", "kvp_status_word", "kvp_last_launch", "kvp_tune",
             "kvp_kernel_times", "kvp_last_error", "kvp_compose_noalloc"]
 
@@ -220,8 +223,9 @@ class Context:
                                                  ctypes.byref(out)))
         return out.value
 
-    def assemble(self, items: Sequence[Sequence[Tuple[int, int]]], flags: int = REBASE, stream=None):
-        """items[b] = [(packet_id, adapter_id), ...].  Returns (assembly_id, prefix_len list)."""
+    def assemble(self, items: Sequence[Sequence[Tuple[int, int]]], flags: int = REBASE, stream=None, pos_base=None):
+        """items[b] = [(packet_id, adapter_id), ...].  Returns (assembly_id, prefix_len list).
+        pos_base (one position per request) -> ``kvp_assemble_at``: this rank's part of a sharded request."""
         offs, pids, aids = [0], [], []
         for it in items:
             for pid, aid in it:
@@ -231,9 +235,20 @@ class Context:
         B = len(items)
         plen = (ctypes.c_int32 * max(1, B))()
         aid = ctypes.c_int32(-1)
-        self._check(self._L.kvp_assemble(self._h, B, _i32_array(offs), _i32_array(pids), _i32_array(aids), flags,
-                                         self._stream(stream), plen, ctypes.byref(aid)))
+        if pos_base is not None:
+            self._check(self._L.kvp_assemble_at(self._h, B, _i32_array(offs), _i32_array(pids), _i32_array(aids),
+                                                _i32_array(list(pos_base)), flags, self._stream(stream), plen, ctypes.byref(aid)))
+        else:
+            self._check(self._L.kvp_assemble(self._h, B, _i32_array(offs), _i32_array(pids), _i32_array(aids), flags,
+                                             self._stream(stream), plen, ctypes.byref(aid)))
         return aid.value, [int(plen[b]) for b in range(B)]
+
+    def partial_bytes(self, batch: int, q_len: int) -> int:
+        return int(self._L.kvp_partial_bytes(self._h, batch, q_len))
+
+    def merge_partials(self, parts, n_parts: int, batch: int, q_len: int, out, lse=None, stream=None):
+        self._check(self._L.kvp_merge_partials(self._h, _ptr(parts), n_parts, batch, q_len, _ptr(out), _ptr(lse),
+                                               self._stream(stream)))
 
     def query_prefill(self, assembly_id: int, layer: int, q, k_new, v_new, q_len: int, out, lse=None,
                       flags: int = 0, stream=None):

@@ -39,7 +39,7 @@ sched_layout schedule_layout(const kvp_config *c)
     const int64_t tiles_q = ((int64_t)group * c->max_query_tokens + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
     const int64_t units = (int64_t)c->max_batch * c->n_kv_heads * tiles_q;
     s.max_works = (int32_t)std::min<int64_t>(units + kMaxCtas, 1 << 24);
-    s.max_merges = 2 * kMaxCtas + 8;
+    s.max_merges = 2 * kMaxCtas + 8 + (int32_t)std::min<int64_t>(units, KVP_MAX_SPLIT_UNITS);   // every unit has one with KVP_PARTIAL
     s.works = round_up(4 * (kMaxCtas + 1), 256);
     s.merges = round_up(s.works + sizeof(kvp_work) * (uint64_t)s.max_works, 256);
     s.total = round_up(s.merges + sizeof(kvp_merge_item) * (uint64_t)s.max_merges, 256);
@@ -215,11 +215,14 @@ struct schedule_t {
 
 // q_lens: nullptr, or one query length per request (<= q_len, the stride of the padded tensors); a request's
 // work records and merge items then carry its own length.
+// opts: KVP_PARTIAL - every unit writes partial slots and gets merge items (even with one piece or none);
+// KVP_SKIP_QUERY_BLOCK - a unit's range starts behind the causal tiles of the query's own keys.
 int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int q_len, int q_pos0, const int32_t *q_lens,
-                      schedule_t &out)
+                      uint32_t opts, schedule_t &out)
 {
     const kvp_shape &sh = ctx->shape;
-    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces, q_len; };
+    const bool force_partial = (opts & KVP_PARTIAL) != 0, skip_tail = (opts & KVP_SKIP_QUERY_BLOCK) != 0;
+    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces, q_len, t_first; };
     std::vector<unit_t> units;
     const int max_rows = sh.group * q_len;
     int64_t total = 0;
@@ -238,10 +241,12 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 u.b = b; u.hk = hk; u.row_base = row_base;
                 u.mode = (n_rows - row_base <= KVP_TILE_ROWS) ? 1 : 0;
                 const int last = std::min(n_rows - 1, row_base + (u.mode ? 1 : 2) * KVP_TILE_ROWS - 1);
-                u.n_all = (q_pos0 + last / sh.group) / KVP_TILE_KEYS + 1 + n_prefix;
+                const int n_tail = (q_pos0 + last / sh.group) / KVP_TILE_KEYS + 1;
+                u.n_all = n_tail + n_prefix;
+                u.t_first = skip_tail ? n_tail : 0;
                 u.first_piece = u.n_pieces = 0;
                 units.push_back(u);
-                total += (int64_t)u.n_all * (u.mode ? 1 : 2) + kPieceCost;
+                total += (int64_t)(u.n_all - u.t_first) * (u.mode ? 1 : 2) + kPieceCost;
             }
         }
     int G = std::min(ctx->sm_count, kMaxCtas);
@@ -257,7 +262,8 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     auto fill = [&](size_t u_begin, size_t u_end, int64_t budget, std::vector<cut_t> *rec) -> int {
         int used = 0;
         size_t u = u_begin;
-        int32_t t = 0;
+        while (u < u_end && units[u].n_all == units[u].t_first) ++u;      // units without a key tile get no piece
+        int32_t t = u < u_end ? units[u].t_first : 0;
         while (u < u_end) {
             ++used;
             if (rec) rec->push_back({(int32_t)u, t});
@@ -267,7 +273,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 const int32_t left = units[u].n_all - t;
                 const int64_t room = budget - cost - kPieceCost;
                 int32_t take = (int32_t)std::min<int64_t>(left, room > 0 ? (room + w - 1) / w : 0);
-                if (no_split) take = (t == 0 && (2 * take >= left || cost == 0)) ? left : 0;
+                if (no_split) take = (t == units[u].t_first && (2 * take >= left || cost == 0)) ? left : 0;
                 if (left - take < 2) take = left;                 // do not leave a sliver behind
                 if (take < 2 && take < left) take = 0;
                 if (take == 0) {
@@ -277,7 +283,11 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 }
                 cost += kPieceCost + (int64_t)take * w;
                 t += take;
-                if (t == units[u].n_all) { ++u; t = 0; }
+                if (t == units[u].n_all) {
+                    ++u;
+                    while (u < u_end && units[u].n_all == units[u].t_first) ++u;
+                    t = u < u_end ? units[u].t_first : 0;
+                }
                 if (cost >= budget) break;
             }
         }
@@ -301,7 +311,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
             rb_begin.push_back(u);
             rb_weight.push_back(0);
         }
-        rb_weight.back() += (int64_t)units[u].n_all * (units[u].mode ? 1 : 2) + kPieceCost;
+        rb_weight.back() += (int64_t)(units[u].n_all - units[u].t_first) * (units[u].mode ? 1 : 2) + kPieceCost;
     }
     rb_begin.push_back(units.size());
     const int n_rb = (int)rb_weight.size();
@@ -340,7 +350,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
         const cut_t a = cuts[c], z = cuts[c + 1];
         cta_rec rec;
         for (int32_t u = a.u; u <= z.u && u < (int32_t)units.size(); ++u) {
-            const int32_t lo = (u == a.u) ? a.t : 0;
+            const int32_t lo = (u == a.u) ? a.t : units[u].t_first;
             const int32_t hi = (u == z.u) ? z.t : units[u].n_all;
             if (hi <= lo) continue;
             kvp_work w;
@@ -381,7 +391,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     int32_t n_slots = 0, max_pieces = 1;
     for (size_t ui = 0; ui < units.size(); ++ui) {
         const unit_t &u = units[ui];
-        if (u.n_pieces <= 1) continue;
+        if (u.n_pieces <= 1 && !force_partial) continue;
         max_pieces = std::max(max_pieces, u.n_pieces);
         const int32_t base = n_slots;
         for (int i = 0; i < u.n_pieces; ++i) {
@@ -414,10 +424,10 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
 }
 
 int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer, int q_len, int q_pos0, const int32_t *q_lens,
-                       cudaStream_t st)
+                       uint32_t opts, cudaStream_t st)
 {
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, as, layer, q_len, q_pos0, q_lens, sc);
+    const int32_t rc = plan_schedule(ctx, as, layer, q_len, q_pos0, q_lens, opts, sc);
     if (rc != KVP_OK) return rc;
     const std::vector<int32_t> &cta_begin = sc.cta_begin;
     const std::vector<kvp_work> &works = sc.works;
@@ -442,6 +452,7 @@ int32_t build_schedule(kvp_ctx *ctx, kvp_assembly_host &as, int slot, int layer,
     ss.q_len = q_len;
     ss.q_lens.assign(q_lens ? q_lens : nullptr, q_lens ? q_lens + as.batch : nullptr);
     ss.q_pos0 = q_pos0;
+    ss.opts = opts;
     ss.ctas = n_ctas;
     ss.works = (int32_t)works.size();
     ss.merges = (int32_t)merges.size();
@@ -765,9 +776,9 @@ int32_t kvp_register_adapter(kvp_ctx *ctx, const void *hk, const void *hv, int32
     return KVP_OK;
 }
 
-int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, const int32_t *packet_ids,
-                     const int32_t *adapter_ids, uint32_t flags, void *stream, int32_t *prefix_len,
-                     int32_t *assembly_id)
+static int32_t assemble_impl(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, const int32_t *packet_ids,
+                             const int32_t *adapter_ids, const int32_t *pos_base, uint32_t flags, void *stream,
+                             int32_t *prefix_len, int32_t *assembly_id)
 {
     if (!ctx) return KVP_ERR_INVALID;
     if (!slot_offsets || !packet_ids || !adapter_ids || !prefix_len || !assembly_id || batch <= 0)
@@ -792,6 +803,10 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
     kvp_assembly_host as;
     as.flags = flags;
     as.batch = batch;
+    as.shard = pos_base != nullptr;
+    if (pos_base)
+        for (int b = 0; b < batch; ++b)
+            if (pos_base[b] < 0) return fail(ctx, KVP_ERR_INVALID, "assemble_at: pos_base[%d] < 0", b);
     // packets that still wait in host memory are brought in now, layer by layer, on the context's own stream
     std::vector<int32_t> to_load;
     bool host_origin = false;
@@ -842,7 +857,7 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
                 e.src_row0 = sg->row0;
                 e.len = sg->n;
                 e.dst_pos0 = (int32_t)t;
-                e.delta = rebase ? (int32_t)(t - sg->pos0) : 0;
+                e.delta = rebase ? (int32_t)(t + (pos_base ? pos_base[b] : 0) - sg->pos0) : 0;
                 auto f = rope_of.find(e.delta);
                 if (f == rope_of.end()) {
                     f = rope_of.emplace(e.delta, (int32_t)rope_delta.size()).first;
@@ -984,6 +999,22 @@ int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, c
     return KVP_OK;
 }
 
+int32_t kvp_assemble(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, const int32_t *packet_ids,
+                     const int32_t *adapter_ids, uint32_t flags, void *stream, int32_t *prefix_len,
+                     int32_t *assembly_id)
+{
+    return assemble_impl(ctx, batch, slot_offsets, packet_ids, adapter_ids, nullptr, flags, stream, prefix_len, assembly_id);
+}
+
+int32_t kvp_assemble_at(kvp_ctx *ctx, int32_t batch, const int32_t *slot_offsets, const int32_t *packet_ids,
+                        const int32_t *adapter_ids, const int32_t *pos_base, uint32_t flags, void *stream,
+                        int32_t *prefix_len, int32_t *assembly_id)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (!pos_base) return fail(ctx, KVP_ERR_INVALID, "assemble_at: pos_base is null");
+    return assemble_impl(ctx, batch, slot_offsets, packet_ids, adapter_ids, pos_base, flags, stream, prefix_len, assembly_id);
+}
+
 int32_t kvp_export_plan(kvp_ctx *ctx, int32_t assembly_id, int32_t b, int32_t *src_row, int32_t *delta,
                         int32_t *seg_table, int32_t *n_segments)
 {
@@ -1040,7 +1071,13 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "query_prefill: unknown assembly %d", assembly_id);
     if (!q || !k_new || !v_new || !out || layer < 0 || layer >= ctx->cfg.n_layers || q_len <= 0)
         return fail(ctx, KVP_ERR_INVALID, "query_prefill: bad arguments");
-    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE | KVP_CONTINUE | KVP_PRECISE_QK)) return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    if (flags & ~(uint32_t)(KVP_ROPE_QUERY | KVP_FORCE_SIMPLE | KVP_CONTINUE | KVP_PRECISE_QK | KVP_PARTIAL | KVP_SKIP_QUERY_BLOCK))
+        return fail(ctx, KVP_ERR_INVALID, "query_prefill: unknown flags");
+    const uint32_t part_opts = flags & (uint32_t)(KVP_PARTIAL | KVP_SKIP_QUERY_BLOCK);
+    if ((flags & KVP_SKIP_QUERY_BLOCK) && !(flags & KVP_PARTIAL))
+        return fail(ctx, KVP_ERR_INVALID, "query_prefill: KVP_SKIP_QUERY_BLOCK needs KVP_PARTIAL");
+    if (part_opts && ((flags & (KVP_CONTINUE | KVP_ROPE_QUERY | KVP_FORCE_SIMPLE)) || q_lens || !ctx->have_tma))
+        return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: KVP_PARTIAL runs on the tcgen05 kernel only, without KVP_CONTINUE, KVP_ROPE_QUERY or per-request lengths");
     {
         // every kernel reads whole elements; the tcgen05 path moves q and out 16 bytes at a time
         const uintptr_t all = (uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)out;
@@ -1061,6 +1098,9 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
     if (as.waits_loads) KVP_CUDA(ctx, cudaStreamWaitEvent(st, ctx->load_done[layer], 0));   // this layer's documents have landed
     const kvp_plan_dev plan = plan_dev(ctx, slot);
     const int rope_query = (flags & KVP_ROPE_QUERY) ? 1 : 0;
+    if (rope_query && as.shard)
+        return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill: KVP_ROPE_QUERY on an assembly made by kvp_assemble_at (the query's position is not prefix_len)");
+    const bool skip_block = (flags & KVP_SKIP_QUERY_BLOCK) != 0;
     const double *inv_freq_dev = reinterpret_cast<const double *>((char *)ctx->cfg.workspace + 256);
 
     int launches = 0;
@@ -1070,21 +1110,21 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
     kvp_attn2_args a;
     a.tail_direct = 0;
     a.precise = (flags & KVP_PRECISE_QK) ? 1 : 0;
-    if (fast && ctx->fused_append && !rope_query && q_pos0 == 0 &&
+    if (fast && ctx->fused_append && !rope_query && q_pos0 == 0 && !skip_block &&
         (((uintptr_t)k_new | (uintptr_t)v_new) & 15) == 0 &&
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_knew, k_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch) &&
         make_query_tensor_map((encode_tiled_fn)ctx->encode_tiled, &a.tm_vnew, v_new, sh.head_dim, sh.n_kv_heads, q_len, as.batch))
         a.tail_direct = 1;
     if (q_lens && !a.tail_direct)
         return fail(ctx, KVP_ERR_UNSUPPORTED, "query_prefill_ragged: needs the tcgen05 kernel with its own append (bf16, head_dim 128, 16-byte aligned k_new / v_new)");
-    if (!a.tail_direct) {
+    if (!a.tail_direct && !skip_block) {
         KVP_CUDA(ctx, kvp_launch_append(sh, plan, as.batch, q_len, q_pos0, q, k_new, v_new, ctx->slot_k[slot], ctx->slot_v[slot],
                                         layer, rope_query, inv_freq_dev, ctx->q_scratch, st));
         ++launches;
     }
     const void *q_used = rope_query ? (const void *)ctx->q_scratch : q;
     as.last_q_len = q_len;
-    as.appended[layer] = q_lens ? 0 : q_pos0 + q_len;       // after a ragged call the rows behind the prefixes differ per request
+    as.appended[layer] = (q_lens || skip_block) ? 0 : q_pos0 + q_len;       // after a ragged call the rows behind the prefixes differ per request
     if (q_lens) as.ragged = true;
 
     int32_t ctas = 0, splits = 1;
@@ -1101,8 +1141,9 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
         const bool same_lens = q_lens ? (as.sched[li].q_lens.size() == (size_t)as.batch &&
                                           std::equal(q_lens, q_lens + as.batch, as.sched[li].q_lens.begin()))
                                        : as.sched[li].q_lens.empty();
-        if (as.sched[li].q_len != q_len || as.sched[li].q_pos0 != q_pos0 || as.sched[li].ctas == 0 || !same_lens) {
-            const int32_t rc = build_schedule(ctx, as, slot, layer, q_len, q_pos0, q_lens, st);
+        if (as.sched[li].q_len != q_len || as.sched[li].q_pos0 != q_pos0 || as.sched[li].ctas == 0 || !same_lens ||
+            as.sched[li].opts != part_opts) {
+            const int32_t rc = build_schedule(ctx, as, slot, layer, q_len, q_pos0, q_lens, part_opts, st);
             if (rc != KVP_OK) return rc;
         }
         const kvp_assembly_host::sched_state &ss = as.sched[li];
@@ -1124,14 +1165,19 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
         a.partial_o = ctx->partial_o;
         a.partial_ml = ctx->partial_ml;
         a.status = ctx->status_dev;
-        KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
-        KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot], ctx->tm_ws_v[slot], st));
-        KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
-        ++launches;
+        if (ss.ctas > 0) {                                         // (a rank may hold no key of any request)
+            KVP_CUDA(ctx, time_edge(ctx, 0, 0, st));
+            KVP_CUDA(ctx, kvp_launch_attn_sm100(sh, a, ctx->tm_pool_k, ctx->tm_pool_v, ctx->tm_ws_k[slot], ctx->tm_ws_v[slot], st));
+            KVP_CUDA(ctx, time_edge(ctx, 0, 1, st));
+            ++launches;
+        }
         if (ss.merges > 0) {
+            const bool partial = (flags & KVP_PARTIAL) != 0;
+            const int64_t n_rt = ((int64_t)sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
             KVP_CUDA(ctx, kvp_launch_merge_list(sh, q_len, ss.merges,
                                                 reinterpret_cast<const kvp_merge_item *>(sd + ctx->sched_off_merges),
-                                                ctx->partial_o, ctx->partial_ml, out, lse, st));
+                                                ctx->partial_o, ctx->partial_ml, out, lse, partial ? out : nullptr,
+                                                (int64_t)as.batch * sh.n_kv_heads * n_rt, st));
             ++launches;
         }
         ctas = ss.ctas;
@@ -1162,6 +1208,29 @@ int32_t kvp_query_prefill_ragged(kvp_ctx *ctx, int32_t assembly_id, int32_t laye
         if (q_lens[b] < 1 || q_lens[b] > q_len_max)
             return fail(ctx, KVP_ERR_INVALID, "query_prefill_ragged: q_lens[%d] = %d outside [1, %d]", b, q_lens[b], q_len_max);
     return query_prefill_impl(ctx, assembly_id, layer, q, k_new, v_new, q_len_max, q_lens, 0, out, lse, stream);
+}
+
+uint64_t kvp_partial_bytes(kvp_ctx *ctx, int32_t batch, int32_t q_len)
+{
+    if (!ctx || batch <= 0 || q_len <= 0) return 0;
+    const kvp_shape &sh = ctx->shape;
+    const uint64_t n_rt = ((uint64_t)sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
+    return (uint64_t)batch * sh.n_kv_heads * n_rt * (KVP_TILE_ROWS * ((uint64_t)sh.head_dim * 4 + 8));
+}
+
+int32_t kvp_merge_partials(kvp_ctx *ctx, const void *parts, int32_t n_parts, int32_t batch, int32_t q_len, void *out,
+                           float *lse, void *stream)
+{
+    if (!ctx) return KVP_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, KVP_ERR_STATE, "merge_partials: host-only context");
+    if (!parts || !out || n_parts <= 0 || batch <= 0 || q_len <= 0 || (((uintptr_t)parts | (uintptr_t)out) & 15) || ((uintptr_t)lse & 3))
+        return fail(ctx, KVP_ERR_INVALID, "merge_partials: bad arguments (parts and out must be 16-byte aligned)");
+    if (!ctx->have_tma) return fail(ctx, KVP_ERR_UNSUPPORTED, "merge_partials: bf16, head_dim 128, sm_100 only");
+    if (batch > ctx->cfg.max_batch || q_len > ctx->cfg.max_query_tokens)
+        return fail(ctx, KVP_ERR_CAPACITY, "merge_partials: batch or q_len beyond the context's maxima");
+    KVP_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    KVP_CUDA(ctx, kvp_launch_merge_ranks(ctx->shape, batch, q_len, parts, n_parts, out, lse, (cudaStream_t)stream));
+    return KVP_OK;
 }
 
 int32_t kvp_segment_mass(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q, const float *lse,
@@ -1222,7 +1291,7 @@ int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, in
     if (slot < 0) return fail(ctx, KVP_ERR_NOT_FOUND, "export_schedule: unknown assembly %d", assembly_id);
     if (q_len <= 0 || q_len > ctx->cfg.max_query_tokens) return fail(ctx, KVP_ERR_INVALID, "export_schedule: bad q_len");
     schedule_t sc;
-    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], 0, q_len, 0, nullptr, sc);
+    const int32_t rc = plan_schedule(ctx, ctx->slots[slot], 0, q_len, 0, nullptr, 0, sc);
     if (rc != KVP_OK) return rc;
     counts[0] = sc.n_ctas;
     counts[1] = (int32_t)sc.works.size();

@@ -1131,43 +1131,56 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_pool_k, const __grid_co
     }
 }
 
-// ---- merge of the partial slots of split units ------------------------------------------------------------
-// Partials hold, per (slot, row): un-normalised O (fp32, stored [32 float4 columns][128 rows]), the
-// running max m of the raw scores and the sum l of exp2((s - m) * c).  Block = 32 rows of one merge
-// item; lanes run along rows while reading (coalesced), the result is turned through shared memory so
-// that the bf16 output rows are written 256 contiguous bytes at a time.  Grid (merge item, 4).
-__global__ void __launch_bounds__(256)
-merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q, int group, float scale,
-                  const float *__restrict__ part_o, const float2 *__restrict__ part_ml,
-                  __nv_bfloat16 *__restrict__ out, float *__restrict__ lse)
+// ---- merge of partial results -------------------------------------------------------------------------------
+// A partial holds, per 128-row query tile: un-normalised O (fp32, stored [32 float4 columns][128 rows]), the
+// running max m of the raw scores and the sum l of exp2((s - m) * c).  Block = 32 rows of one query tile; lanes
+// run along rows while reading (coalesced).  The partials of a tile are `n` blocks `stride` apart (the slots of
+// a unit cut into pieces: consecutive; the same tile on every rank of a prefix-sharded request: one rank buffer
+// apart).  The result is either final - normalised, turned through shared memory so that bf16 output rows are
+// written 256 contiguous bytes at a time - or again a partial, in the canonical order of a rank buffer
+// [request][kv head][row tile] (KVP_PARTIAL: what a rank hands to the exchange).
+struct MergeOut {
+    __nv_bfloat16 *out;         // final: [batch][q_len][n_q][128]
+    float *lse;
+    float4 *part_o;             // or partial: [tiles][32][128] float4 ...
+    float2 *part_ml;            // ... and [tiles][128] (m, l)
+};
+
+__device__ __forceinline__ void merge_tile(int b, int hk, int row_base, int item_q_len, const float4 *po, const float2 *pml,
+                                           int n, long long stride_o, long long stride_ml, int q_len, int n_q, int n_kv,
+                                           int group, float scale, const MergeOut &mo)
 {
     __shared__ uint2 tile[32][33];
-    const kvp_merge_item mi = merges[blockIdx.x];
     const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5;
     const int row = blockIdx.y * 32 + lane;                     // row of the 128-row query tile
-    const int n_rows = group * (mi.pad[0] ? mi.pad[0] : q_len);         // q_len stays the stride of the padded tensors
+    const int n_rows = group * (item_q_len ? item_q_len : q_len);       // q_len stays the stride of the padded tensors
     const float c2 = scale * 1.4426950408889634f;
-    const float4 *po = reinterpret_cast<const float4 *>(part_o);
     float M = -INFINITY;
-    for (int s = 0; s < mi.n_slots; ++s) {
-        const float2 ml = part_ml[(long long)(mi.slot0 + s) * KVP_TILE_ROWS + row];
+    for (int s = 0; s < n; ++s) {
+        const float2 ml = pml[s * stride_ml + row];
         if (ml.y > 0.f) M = fmaxf(M, ml.x);
     }
     float L = 0.f;
     float4 o[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < mi.n_slots; ++s) {
-        const long long slot = mi.slot0 + s;
-        const float2 ml = part_ml[slot * KVP_TILE_ROWS + row];
+    for (int s = 0; s < n; ++s) {
+        const float2 ml = pml[s * stride_ml + row];
         if (!(ml.y > 0.f)) continue;                            // an empty partial: nothing was visible to this row
         const float w = exp2f((ml.x - M) * c2);
         L += w * ml.y;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const float4 a = po[(slot * 32 + wv + 8 * j) * KVP_TILE_ROWS + row];
+            const float4 a = po[s * stride_o + (wv + 8 * j) * KVP_TILE_ROWS + row];
             o[j].x += w * a.x; o[j].y += w * a.y; o[j].z += w * a.z; o[j].w += w * a.w;
         }
+    }
+    if (mo.part_o != nullptr) {                                 // stays a partial: un-normalised, against the max M
+        const long long c = ((long long)b * n_kv + hk) * ((group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS) + row_base / KVP_TILE_ROWS;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mo.part_o[(c * 32 + wv + 8 * j) * KVP_TILE_ROWS + row] = o[j];
+        if (wv == 0) mo.part_ml[c * KVP_TILE_ROWS + row] = make_float2(L > 0.f ? M : -1e30f, L);
+        return;
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll
@@ -1177,20 +1190,44 @@ merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q,
         u.y = pack_bf16(o[j].z * inv, o[j].w * inv);
         tile[lane][wv + 8 * j] = u;
     }
-    const int r = mi.row_base + row;
-    if (wv == 0 && r < n_rows && lse != nullptr)
-        lse[((long long)mi.b * n_q + mi.hk * group + r % group) * q_len + r / group] = M * scale + logf(L);
+    const int r = row_base + row;
+    if (wv == 0 && r < n_rows && mo.lse != nullptr)
+        mo.lse[((long long)b * n_q + hk * group + r % group) * q_len + r / group] = M * scale + logf(L);
     __syncthreads();
     // 8 threads per output row, 32 bytes each
     const int orow = threadIdx.x >> 3, j8 = threadIdx.x & 7;
-    const int r2 = mi.row_base + blockIdx.y * 32 + orow;
+    const int r2 = row_base + blockIdx.y * 32 + orow;
     if (r2 < n_rows) {
-        const int i = r2 / group, h = mi.hk * group + r2 % group;
-        uint4 *dst = reinterpret_cast<uint4 *>(out + (((long long)mi.b * q_len + i) * n_q + h) * 128) + 2 * j8;
+        const int i = r2 / group, h = hk * group + r2 % group;
+        uint4 *dst = reinterpret_cast<uint4 *>(mo.out + (((long long)b * q_len + i) * n_q + h) * 128) + 2 * j8;
         const uint2 a0 = tile[orow][4 * j8], a1 = tile[orow][4 * j8 + 1], a2 = tile[orow][4 * j8 + 2], a3 = tile[orow][4 * j8 + 3];
         dst[0] = make_uint4(a0.x, a0.y, a1.x, a1.y);
         dst[1] = make_uint4(a2.x, a2.y, a3.x, a3.y);
     }
+}
+
+// The partial slots of the units of one launch.  Grid (merge item, 4).
+__global__ void __launch_bounds__(256)
+merge_list_kernel(const kvp_merge_item *__restrict__ merges, int q_len, int n_q, int n_kv, int group, float scale,
+                  const float *__restrict__ part_o, const float2 *__restrict__ part_ml, MergeOut mo)
+{
+    const kvp_merge_item mi = merges[blockIdx.x];
+    merge_tile(mi.b, mi.hk, mi.row_base, mi.pad[0], reinterpret_cast<const float4 *>(part_o) + (long long)mi.slot0 * (32 * KVP_TILE_ROWS),
+               part_ml + (long long)mi.slot0 * KVP_TILE_ROWS, mi.n_slots, 32 * KVP_TILE_ROWS, KVP_TILE_ROWS, q_len, n_q, n_kv,
+               group, scale, mo);
+}
+
+// The rank buffers of a prefix-sharded request, `n_parts` of them `part_bytes` apart.  Grid (query tile, 4), query
+// tiles in the canonical order [request][kv head][row tile].
+__global__ void __launch_bounds__(256)
+merge_ranks_kernel(const char *__restrict__ parts, int n_parts, long long part_bytes, long long ml_offset, int n_rt, int q_len,
+                   int n_q, int n_kv, int group, float scale, MergeOut mo)
+{
+    const int c = blockIdx.x;
+    const int rt = c % n_rt, hk = (c / n_rt) % n_kv, b = c / (n_rt * n_kv);
+    merge_tile(b, hk, rt * KVP_TILE_ROWS, 0, reinterpret_cast<const float4 *>(parts) + (long long)c * (32 * KVP_TILE_ROWS),
+               reinterpret_cast<const float2 *>(parts + ml_offset) + (long long)c * KVP_TILE_ROWS, n_parts, part_bytes / 16,
+               part_bytes / 8, q_len, n_q, n_kv, group, scale, mo);
 }
 
 }  // namespace
@@ -1239,10 +1276,35 @@ cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, 
 
 cudaError_t kvp_launch_merge_list(const kvp_shape &sh, int32_t q_len, int32_t n_merges, const kvp_merge_item *merges,
                                   const float *partial_o, const float2 *partial_ml, void *out, float *lse,
-                                  cudaStream_t st)
+                                  void *part_out, int64_t part_tiles, cudaStream_t st)
 {
     if (n_merges <= 0) return cudaSuccess;
-    merge_list_kernel<<<dim3(n_merges, KVP_TILE_ROWS / 32), 256, 0, st>>>(merges, q_len, sh.n_q_heads, sh.group, sh.scale,
-                                                                        partial_o, partial_ml, (__nv_bfloat16 *)out, lse);
+    MergeOut mo;
+    mo.out = (__nv_bfloat16 *)out;
+    mo.lse = lse;
+    mo.part_o = nullptr;
+    mo.part_ml = nullptr;
+    if (part_out != nullptr) {                                   // KVP_PARTIAL: `out` stays untouched
+        mo.part_o = reinterpret_cast<float4 *>(part_out);
+        mo.part_ml = reinterpret_cast<float2 *>((char *)part_out + (uint64_t)part_tiles * (32ull * KVP_TILE_ROWS * 16));
+    }
+    merge_list_kernel<<<dim3(n_merges, KVP_TILE_ROWS / 32), 256, 0, st>>>(merges, q_len, sh.n_q_heads, sh.n_kv_heads, sh.group,
+                                                                        sh.scale, partial_o, partial_ml, mo);
+    return cudaGetLastError();
+}
+
+cudaError_t kvp_launch_merge_ranks(const kvp_shape &sh, int32_t batch, int32_t q_len, const void *parts, int32_t n_parts,
+                                   void *out, float *lse, cudaStream_t st)
+{
+    const int n_rt = (sh.group * q_len + KVP_TILE_ROWS - 1) / KVP_TILE_ROWS;
+    const uint64_t tiles = (uint64_t)batch * sh.n_kv_heads * n_rt;
+    MergeOut mo;
+    mo.out = (__nv_bfloat16 *)out;
+    mo.lse = lse;
+    mo.part_o = nullptr;
+    mo.part_ml = nullptr;
+    merge_ranks_kernel<<<dim3((unsigned)tiles, KVP_TILE_ROWS / 32), 256, 0, st>>>(
+        (const char *)parts, n_parts, (long long)(tiles * (32ull * KVP_TILE_ROWS * 16 + KVP_TILE_ROWS * 8)),
+        (long long)(tiles * (32ull * KVP_TILE_ROWS * 16)), n_rt, q_len, sh.n_q_heads, sh.n_kv_heads, sh.group, sh.scale, mo);
     return cudaGetLastError();
 }

@@ -116,11 +116,12 @@ struct kvp_assembly_host {
     int32_t item_stride = 0;               // batch when the assembly has a tile list per (layer, kv head) (compressed packets)
     int32_t last_q_len = 0;
     std::vector<int32_t> appended;         // per layer: query rows appended so far (KVP_CONTINUE)
+    bool shard = false;                    // made by kvp_assemble_at: positions start at a caller-given base
     bool ragged = false;                   // a kvp_query_prefill_ragged call has appended a different number of rows per request
     bool waits_loads = false;              // uses packets that came from host memory: wait for the layer's load event
     // work lists of the two-stream kernel (one, or one per layer when the tile lists differ per layer), each
     // built for q_len query tokens at offset q_pos0 (q_len 0 = none yet)
-    struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; std::vector<int32_t> q_lens; };
+    struct sched_state { int32_t q_len = 0, q_pos0 = 0, ctas = 0, works = 0, merges = 0, slots = 0; uint32_t opts = 0; std::vector<int32_t> q_lens; };
     std::vector<sched_state> sched;
 };
 
@@ -226,6 +227,10 @@ cudaError_t kvp_attn_sm100_prepare(void);
 cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, const CUtensorMap &tm_pool_k,
                                   const CUtensorMap &tm_pool_v, const CUtensorMap &tm_ws_k,
                                   const CUtensorMap &tm_ws_v, cudaStream_t st);
+// part_out != nullptr: the merged tiles stay partials and go to a rank buffer of part_tiles query tiles
 cudaError_t kvp_launch_merge_list(const kvp_shape &sh, int32_t q_len, int32_t n_merges, const kvp_merge_item *merges,
                                   const float *partial_o, const float2 *partial_ml, void *out, float *lse,
-                                  cudaStream_t st);
+                                  void *part_out, int64_t part_tiles, cudaStream_t st);
+// n_parts rank buffers back to back -> final output rows
+cudaError_t kvp_launch_merge_ranks(const kvp_shape &sh, int32_t batch, int32_t q_len, const void *parts, int32_t n_parts,
+                                   void *out, float *lse, cudaStream_t st);

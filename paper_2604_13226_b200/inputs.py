@@ -153,6 +153,33 @@ class Workload:
         return self.q[layer], self.k_new[layer], self.v_new[layer]
 
 
+def shard_workload(wl: Workload, rank: int, world: int):
+    """Rank ``rank``'s part of a workload whose requests are sharded by prefix over ``world`` ranks: every
+    request's slot list is cut into ``world`` contiguous parts (slot counts as equal as possible, some possibly
+    empty); the rank keeps only the packets its parts name (local ids in order of first use), all adapters and
+    the whole query.  Returns (sub-workload, pos_base) with pos_base[b] = composed position at which the rank's
+    part of request b starts (the lengths of the slots before it, adapters included)."""
+    local = {}
+    items, pos_base = [], []
+    for it in wl.items:
+        n = len(it)
+        lo, hi = (n * rank) // world, (n * (rank + 1)) // world
+        pos = 0
+        for pid, aid in it[:lo]:
+            pos += wl.packets[pid].n_tokens + (wl.adapters[aid].n_header + wl.adapters[aid].n_trailer if aid >= 0 else 0)
+        pos_base.append(pos)
+        part = []
+        for pid, aid in it[lo:hi]:
+            if pid not in local:
+                local[pid] = len(local)
+            part.append((local[pid], aid))
+        items.append(part)
+    packets = [wl.packets[pid] for pid, _ in sorted(local.items(), key=lambda kv: kv[1])]
+    sub = Workload(wl.shape, packets, wl.adapters, items, wl.q, wl.k_new, wl.v_new, wl.rebase, f"{wl.name}_rank{rank}of{world}",
+                   wl.seed, dict(wl.notes))
+    return sub, pos_base
+
+
 # --------------------------------------------------------------------------------------
 # small, numpy-drawn workloads
 # --------------------------------------------------------------------------------------

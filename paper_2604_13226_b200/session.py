@@ -60,7 +60,7 @@ class Session:
             ws_rows = sum(prefix[b] - sum(lens[pid] for pid, _ in wl.items[b]) for b in range(B)) + B * mq
         self.ctx = kvp.Context(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.dtype, rope_theta=s.rope_theta,
                                rope_pairing=s.rope_pairing, pool_tokens=sum(lens) + ad_tokens + 8,
-                               max_packets=len(lens), max_adapters=max(1, n_adapters), max_batch=B,
+                               max_packets=max(1, len(lens)), max_adapters=max(1, n_adapters), max_batch=B,
                                max_slots=max(1, n_slots), max_prefix_tokens=max(prefix + [1]), max_query_tokens=mq,
                                max_ws_rows=ws_rows + 8, max_assemblies=max_assemblies, device=device,
                                max_compressed=0 if is_dev else sum(1 for p in wl.packets if p.kept is not None))
@@ -108,13 +108,14 @@ class Session:
         self.assembly_id = -1
         self.prefix_len: List[int] = []
 
-    def assemble(self, rebase: Optional[bool] = None, items=None):
+    def assemble(self, rebase: Optional[bool] = None, items=None, pos_base=None):
         flags = 0
         if self.wl.rebase if rebase is None else rebase:
             flags |= kvp.REBASE
         if self.materialize:
             flags |= kvp.MATERIALIZE
-        self.assembly_id, self.prefix_len = self.ctx.assemble(items if items is not None else self.wl.items, flags)
+        self.assembly_id, self.prefix_len = self.ctx.assemble(items if items is not None else self.wl.items, flags,
+                                                              pos_base=pos_base)
         return self.assembly_id, self.prefix_len
 
     def query_tensors(self, layer: int):

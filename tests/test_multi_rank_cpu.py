@@ -59,3 +59,67 @@ def test_two_gloo_ranks_shard_requests_and_reduce_timings(tmp_path):
     assert a["pieces"] >= 1 and b["pieces"] >= 1
     assert a["ms"] == b["ms"] == [11.0, 7.0]                        # maximum over ranks, element-wise
     assert abs(a["value"] - 2 * 2 * 16 / 11.0e-3) < 1e-6 and a["value"] == b["value"]
+
+
+# Prefix sharding (the packets of one request spread over the ranks): every rank plans its part with
+# kvp_assemble_at; the parts must tile the whole request - same segment lengths, the rotation offsets the oracle's
+# composition of the whole request gives, positions shifted by the rank's base - and the ranks agree on the total.
+SHARD_WORKER = r'''
+import json, os, sys
+sys.path.insert(0, os.environ["KVP_ROOT"]); sys.path.insert(0, os.path.join(os.environ["KVP_ROOT"], "tests"))
+import numpy as np
+import torch.distributed as dist
+from oracle import reference as orc
+from paper_2604_13226_b200 import binding as kvp, inputs as gen
+from helpers import make_store
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", rank=rank, world_size=world)
+shape = gen.ModelShape(1, 4, 2, 64, "f32", 10000.0, 0)
+lens = [40, 130, 7, 64, 90]
+items = [[(0, 0), (1, 0), (2, -1), (3, 0), (4, 0)], [(4, 0), (0, 0), (1, -1)], [(2, 0)]]
+wl = gen.make_workload(shape, lens, items, q_len=4, n_header=3, n_trailer=5, seed=9, packet_pos0=[0, 11, 0, 500, 2])
+sub, pos_base = gen.shard_workload(wl, rank, world)
+ctx = kvp.Context(1, 4, 2, 64, "f32", rope_theta=10000.0, max_packets=8, max_adapters=1, max_batch=3, max_slots=16,
+                  max_prefix_tokens=1024, max_query_tokens=4, max_ws_rows=4096, device=-1)
+for p in sub.packets:
+    ctx.register_packet(None, None, p.n_tokens, p.cache_pos0)
+a = sub.adapters[0]
+ctx.register_adapter(None, None, a.n_header, a.header_pos0, None, None, a.n_trailer, a.trailer_pos0)
+aid, plen = ctx.assemble(sub.items, kvp.REBASE, pos_base=pos_base)
+st = make_store(wl)
+ok = True
+for b in range(wl.batch):
+    whole = orc.compose(st, wl.items[b])
+    segs = whole.segments                                          # [src_row0, len, dst_pos0, delta] of the whole request
+    mine = [s for s in segs if pos_base[b] <= s[2] < pos_base[b] + plen[b]]
+    _, dl, got = ctx.export_plan(aid, b)
+    ok = ok and len(got) == len(mine)
+    for g, m in zip(got, mine):
+        ok = ok and int(g[1]) == int(m[1]) and int(g[3]) == int(m[3]) and int(g[2]) + pos_base[b] == int(m[2])
+    ok = ok and np.array_equal(dl, whole.delta[pos_base[b]:pos_base[b] + plen[b]])
+gathered = [None] * world
+dist.all_gather_object(gathered, (pos_base, plen))
+total = [sum(g[1][b] for g in gathered) for b in range(wl.batch)]
+tiles = all(gathered[r][0][b] + gathered[r][1][b] == gathered[r + 1][0][b] for r in range(world - 1) for b in range(wl.batch))
+print(json.dumps({"rank": rank, "ok": bool(ok), "total": total, "whole": [wl.prefix_len(b) for b in range(wl.batch)],
+                  "tiles": bool(tiles), "partial_bytes": ctx.partial_bytes(3, 4)}))
+dist.destroy_process_group()
+'''
+
+
+def test_two_gloo_ranks_plan_the_parts_of_prefix_sharded_requests(tmp_path):
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER)
+    port = 31500 + os.getpid() % 2000
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port),
+                   KVP_ROOT=ROOT, CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    for p in procs:
+        out, err = p.communicate(timeout=240)
+        assert p.returncode == 0, err[-2000:]
+        d = json.loads(out.strip().splitlines()[-1])
+        assert d["ok"] and d["tiles"] and d["total"] == d["whole"]
+        # 3 requests x 2 kv heads x 1 row tile of 128 packed rows, 64 fp32 columns + (m, l) per row
+        assert d["partial_bytes"] == 3 * 2 * 1 * 128 * (64 * 4 + 8)
