@@ -153,6 +153,52 @@ class Workload:
         return self.q[layer], self.k_new[layer], self.v_new[layer]
 
 
+def draw_kept(packets, keep_rate, seed: int, n_layers: int, n_kv_heads: int, per_head: bool = True) -> None:
+    """Stand-in for an unstructured KV compressor (Section 4.3): packet i keeps about keep_rate[i] of its tokens
+    (None: not pruned), a different seeded random subset per layer and - with per_head - per kv head."""
+    krng = np.random.default_rng(seed + 104729)
+    for i, rate in enumerate(keep_rate):
+        if rate is None:
+            continue
+        n = packets[i].n_tokens
+        kept = []
+        for l in range(n_layers):
+            n_layer = max(1, min(n, int(round(n * rate * krng.uniform(0.7, 1.3)))))
+            row = []
+            for h in range(n_kv_heads):
+                n_h = max(1, min(n, int(round(n_layer * krng.uniform(0.6, 1.0))))) if per_head else n_layer
+                row.append(np.sort(krng.choice(n, size=n_h, replace=False)).astype(np.int64))
+            kept.append(row)
+        packets[i].kept = kept
+
+
+def wrap_workload(wl: Workload, keep_rate=None, seed: int = 0) -> Workload:
+    """The same requests with every slot's cache stored as ONE wrapped unit  header | document | trailer  (Eq. 2:
+    the form in which the paper computes a packet offline), registered as a packet of its own with no separate
+    adapter.  The fillers must have been cached where the wrapped layout puts them (header right before the
+    document, trailer right behind).  With keep_rate (one rate per slot, in slot order) the wrapped units are
+    pruned as a whole, fillers included - Section 4.3's "KVPacket Normal" setting."""
+    packets, items = [], []
+    for it in wl.items:
+        part = []
+        for pid, aid in it:
+            p = wl.packets[pid]
+            if aid < 0:
+                packets.append(Packet(p.k, p.v, p.cache_pos0))
+            else:
+                a = wl.adapters[aid]
+                assert a.header_pos0 + a.n_header == p.cache_pos0 and a.trailer_pos0 == p.cache_pos0 + p.n_tokens, \
+                    "fillers not cached at the wrapped layout's positions"
+                packets.append(Packet(np.concatenate([a.hk, p.k, a.tk], axis=1), np.concatenate([a.hv, p.v, a.tv], axis=1),
+                                      a.header_pos0))
+            part.append((len(packets) - 1, -1))
+        items.append(part)
+    out = Workload(wl.shape, packets, [], items, wl.q, wl.k_new, wl.v_new, wl.rebase, wl.name + "_wrapped", wl.seed, dict(wl.notes))
+    if keep_rate is not None:
+        draw_kept(packets, keep_rate, seed, wl.shape.n_layers, wl.shape.n_kv_heads, True)
+    return out
+
+
 def shard_workload(wl: Workload, rank: int, world: int):
     """Rank ``rank``'s part of a workload whose requests are sharded by prefix over ``world`` ranks: every
     request's slot list is cut into ``world`` contiguous parts (slot counts as equal as possible, some possibly
@@ -255,20 +301,7 @@ def make_workload(shape: ModelShape,
                   rebase=rebase, name=name, seed=seed)
     wl.notes["chan_scale"] = chan_scale        # [L][1][Hkv][d] multipliers applied to packet K/V, or None
     if keep_rate is not None:
-        krng = np.random.default_rng(seed + 104729)
-        for i, rate in enumerate(keep_rate):
-            if rate is None:
-                continue
-            n = packets[i].n_tokens
-            kept = []
-            for l in range(L):
-                n_layer = max(1, min(n, int(round(n * rate * krng.uniform(0.7, 1.3)))))
-                row = []
-                for h in range(Hkv):
-                    n_h = max(1, min(n, int(round(n_layer * krng.uniform(0.6, 1.0))))) if keep_per_head else n_layer
-                    row.append(np.sort(krng.choice(n, size=n_h, replace=False)).astype(np.int64))
-                kept.append(row)
-            packets[i].kept = kept
+        draw_kept(packets, keep_rate, seed, L, Hkv, keep_per_head)
     return wl
 
 

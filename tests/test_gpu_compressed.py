@@ -76,3 +76,35 @@ def test_compressed_unsupported_paths_and_validation():
         sess.ctx.assemble(wl.items, kvp.REBASE | kvp.MATERIALIZE)
     assert e.value.code == 5
     sess.close()
+
+
+def test_normal_mode_wrapped_packets_pruned_with_their_fillers():
+    # Section 4.3, "KVPacket Normal": the compressor runs over the whole wrapped cache  header | document | trailer,
+    # so filler tokens are pruned like any other.  A wrapped cache is registered as one packet (no separate
+    # adapter): it is still an opaque unit with one offset.
+    shape = gen.ModelShape(2, 8, 2, 128, "bf16", 500000.0, 0)
+    L, nh, nt = 200, 16, 16
+    base = gen.make_workload(shape, [L, L, L], [[(0, 0), (1, 0)], [(2, 0), (0, 0), (1, 0)]], q_len=24, n_header=nh, n_trailer=nt,
+                             seed=47, packet_pos0=[nh, nh, nh], adapter_pos0=[(0, nh + L)])
+    # (a) unpruned: the wrapped registration composes to the same sequence as packets + shared fillers
+    wrapped = gen.wrap_workload(base)
+    assert [p.n_tokens for p in wrapped.packets] == [nh + L + nt] * 5 and wrapped.adapters == []
+    sess = Session(wrapped)
+    _, plen = sess.assemble()
+    assert plen == [base.prefix_len(b) for b in range(base.batch)]
+    for layer in range(2):
+        out, lse = sess.prefill(layer)
+        check(base, out, lse, layer)                    # the oracle over the ORIGINAL registration
+    sess.close()
+    # (b) pruned as a whole, a different subset per layer and kv head; some units lose most of their fillers
+    pruned = gen.wrap_workload(base, keep_rate=[0.5, 0.3, 0.6, None, 0.1], seed=48)
+    filler = np.r_[0:nh, nh + L:nh + L + nt]
+    assert any(len(np.intersect1d(k, filler)) < (nh + nt) // 2 for p in pruned.packets if p.kept for row in p.kept for k in row)
+    sess = Session(pruned)
+    sess.assemble()
+    for layer in range(2):
+        for flags in (0, kvp.FORCE_SIMPLE):
+            out, lse = sess.prefill(layer, flags)
+            assert sess.ctx.status_word() == 0
+            check(pruned, out, lse, layer)
+    sess.close()
