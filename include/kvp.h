@@ -139,8 +139,10 @@ KVP_API int32_t kvp_register_packet_host(kvp_ctx *ctx, const void *k_host, const
 
 /*
  * Mark a packet registered with kvp_register_packet_host as no longer on the device: the next kvp_assemble
- * that names it copies it in again (into the same pool rows).  The caller must not evict a packet that work
- * already enqueued still reads, other than on the stream it passes to that next kvp_assemble.
+ * that names it copies it in again (into the same pool rows).  Eviction frees no pool capacity: the packet keeps
+ * its rows reserved and no other packet can take them; it only forces the copy to happen again (a packet whose
+ * host copy changed, a transfer to be timed).  The caller must not evict a packet that work already enqueued
+ * still reads, other than on the stream it passes to that next kvp_assemble.
  * Errors: NOT_FOUND, STATE (the packet has no host copy).
  */
 KVP_API int32_t kvp_evict_packet(kvp_ctx *ctx, int32_t packet_id);
@@ -229,8 +231,9 @@ KVP_API int32_t kvp_assemble_at(kvp_ctx *ctx, int32_t batch, const int32_t *slot
  * this call sits at position prefix_len[b] + n + i, attends to the prefix, to those n rows and to this
  * call's tokens <= i, and is appended behind them.  n + q_len may not exceed max_query_tokens.  Without
  * the flag a call starts again at prefix_len[b].  Errors: INVALID, NOT_FOUND, CAPACITY (q_len > max_query_tokens),
- * STATE (host-only context), UNSUPPORTED, CUDA.  Device-side wait timeouts are reported through
- * kvp_status_word after the stream has been synchronised.
+ * STATE (host-only context), UNSUPPORTED, CUDA.  The call returns KVP_OK once the kernels are enqueued: a
+ * device-side wait that ran out (the launch then gave up and its output is not valid) shows only in
+ * kvp_status_word, which a caller that needs to know must read after synchronising the stream.
  */
 KVP_API int32_t kvp_query_prefill(kvp_ctx *ctx, int32_t assembly_id, int32_t layer, const void *q,
                           const void *k_new, const void *v_new, int32_t q_len, uint32_t flags,

@@ -518,6 +518,7 @@ __device__ __forceinline__ void rescale_row(uint32_t s_addr, uint32_t o_addr, fl
             tmem_st32(o_addr + ch * 32, v);
         }
     }
+    if (n_chunks > 0) tc_wait_st();                  // the P chunks this thread stored are read back below
 #pragma unroll 1
     for (int ch = 0; ch < n_chunks; ++ch) {          // 16 columns of packed bf16 pairs per chunk
         asm volatile(
@@ -1156,17 +1157,17 @@ __device__ __forceinline__ void merge_tile(int b, int hk, int row_base, int item
     const int n_rows = group * (item_q_len ? item_q_len : q_len);       // q_len stays the stride of the padded tensors
     const float c2 = scale * 1.4426950408889634f;
     float M = -INFINITY;
-    for (int s = 0; s < n; ++s) {
-        const float2 ml = pml[s * stride_ml + row];
-        if (ml.y > 0.f) M = fmaxf(M, ml.x);
-    }
     float L = 0.f;
     float4 o[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < n; ++s) {
         const float2 ml = pml[s * stride_ml + row];
-        if (!(ml.y > 0.f)) continue;                            // an empty partial: nothing was visible to this row
+        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+    }
+    for (int s = 0; s < n; ++s) {
+        const float2 ml = pml[s * stride_ml + row];
+        if (!(ml.y > 0.f)) continue;                        // an empty partial: nothing was visible to this row
         const float w = exp2f((ml.x - M) * c2);
         L += w * ml.y;
 #pragma unroll

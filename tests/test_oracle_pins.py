@@ -15,17 +15,6 @@ from helpers import make_store, oracle_outputs
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
-def make_store(wl):
-    """Register packets in id order, then adapters in id order (the order every test uses)."""
-    st = orc.Store(wl.shape.dtype)
-    for p in wl.packets:
-        st.register_packet(p.n_tokens, p.cache_pos0, (lambda layer, p=p: (p.k[layer], p.v[layer])))
-    for a in wl.adapters:
-        st.register_adapter(a.n_header, a.header_pos0, a.n_trailer, a.trailer_pos0,
-                            (lambda layer, a=a: (a.hk[layer], a.hv[layer], a.tk[layer], a.tv[layer])))
-    return st
-
-
 def tiny(seed=1, dtype="f32", d=16, Hq=4, Hkv=2, lens=(5, 9, 3), nh=2, nt=3, q_len=4, pairing=0, **kw):
     shape = gen.ModelShape(1, Hq, Hkv, d, dtype, 10000.0, pairing)
     items = [[(p, 0) for p in range(len(lens))]]
