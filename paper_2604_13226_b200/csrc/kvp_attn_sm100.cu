@@ -974,7 +974,7 @@ __device__ __forceinline__ void mma_role(const Params &p, const Cta &c)
                     }
                     if (p.precise && rope != 0) {                // + (rounding remainder of the rotated Q) K^T
                         constexpr uint32_t kRem16 = kTileBytes >> 4;
-#pragma unroll 1
+#pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             constexpr uint32_t kHalf16 = kHalfBytes >> 4;
                             const uint32_t off = (kk >> 2) * kHalf16 + (kk & 3) * 2;
