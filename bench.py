@@ -71,6 +71,10 @@ def make_spec(name: str, seed: int):
     from paper_2604_13226_b200 import inputs as gen
     if name == "config3":
         return gen.spec_config3(seed=seed)
+    if name.startswith("config3:"):                  # the same requests over fewer layers (small profiler captures)
+        s = gen.spec_config3(seed=seed, n_layers=int(name.split(":")[1]))
+        s.name = name.replace(":", "_layers")
+        return s
     if name == "config4":
         return gen.spec_config4(seed=seed)
     if name == "config4_layer":                      # one layer of the Qwen2.5-7B stack: same requests, same raggedness

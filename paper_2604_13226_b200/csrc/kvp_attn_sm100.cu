@@ -737,21 +737,41 @@ __device__ __forceinline__ void producer_role(const Params &p, const Cta &c, con
 }
 
 // ---- append (the two spare warps) -------------------------------------------------------------------------------
-// With tail_direct the attention reads the query block's K/V from the caller's tensors; the piece that starts
-// a (request, kv head) also copies those rows behind the prefix in the workspace, for later calls.  Nothing
-// in this launch waits for the copy.
+// With tail_direct the attention reads the query block's K/V from the caller's tensors; the rows are also copied
+// behind the prefix in the workspace, for later calls.  Every unit copies the query tokens whose first packed row
+// it holds (for its kv head), in the piece that starts the unit, so the copy is spread over all CTAs; four
+// 16-byte words of K and of V are in flight per thread.  Nothing in this launch waits for the copy.
 __device__ __forceinline__ void append_role(const Params &p, const Cta &c, const int t)
 {
     if (!p.tail_direct) return;
     for (int wi = c.item_begin; wi < c.item_end; ++wi) {
         const Work w = load_work(p, wi);
-        if (w.lo != 0 || w.row_base != 0) continue;
-        for (int i = t; i < w.q_len * 16; i += 64) {            // 16-byte words of the rows of this kv head
-            const int row = i >> 4, c4 = i & 15;
-            const long long src = (((long long)w.b * p.q_len + row) * p.n_kv + w.hk) * 16 + c4;
-            const long long dst = ((long long)w.plane * p.ws_rows + w.tail_row0 + row) * 16 + c4;
-            p.ws_k[dst] = __ldg(p.k_new + src);
-            p.ws_v[dst] = __ldg(p.v_new + src);
+        if (w.lo != 0) continue;
+        const int n_rows = p.group * w.q_len;
+        const int row_end = min(n_rows, w.row_base + (w.mode ? KVP_TILE_ROWS : 2 * KVP_TILE_ROWS));
+        const int i0 = (w.row_base + p.group - 1) / p.group, i1 = (row_end + p.group - 1) / p.group;   // tokens [i0, i1)
+        const long long src0 = (((long long)w.b * p.q_len + i0) * p.n_kv + w.hk) * 16;     // 16-byte words; a token's row is 16
+        const long long dst0 = ((long long)w.plane * p.ws_rows + w.tail_row0 + i0) * 16;
+        const int n_words = (i1 - i0) * 16;
+        for (int base = 0; base < n_words; base += 64 * 4) {
+            uint4 k[4], v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + j * 64 + t;
+                if (i < n_words) {
+                    const long long src = src0 + (long long)(i >> 4) * p.n_kv * 16 + (i & 15);
+                    k[j] = __ldg(p.k_new + src);
+                    v[j] = __ldg(p.v_new + src);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + j * 64 + t;
+                if (i < n_words) {
+                    p.ws_k[dst0 + i] = k[j];
+                    p.ws_v[dst0 + i] = v[j];
+                }
+            }
         }
     }
 }
