@@ -1153,6 +1153,7 @@ static int32_t query_prefill_impl(kvp_ctx *ctx, int32_t assembly_id, int32_t lay
         a.ws_k = ctx->slot_k[slot];
         a.ws_v = ctx->slot_v[slot];
         a.plan = plan;
+        a.l2_prefetch = (sh.group * q_len <= 4 * KVP_TILE_ROWS) ? 1 : 0;      // <= 2 units share a (request, kv head)'s K/V
         a.q_len = q_len;
         a.q_pos0 = q_pos0;
         a.layer = layer;

@@ -73,6 +73,9 @@ struct Params {
     // precise: the counter-rotated query is kept as value + rounding remainder (two bf16 tiles per stream, one
     // epoch buffer instead of two) and Q K^T of a rotated tile takes both
     int precise;
+    // l2_prefetch: the K/V tiles of a unit are read by at most two units of the launch, i.e. they come from DRAM
+    // rather than from L2: the TMA warp then asks L2 for each tile a few loads before it fetches it
+    int l2_prefetch;
     const uint4 *k_new, *v_new;
     uint4 *ws_k, *ws_v;
     long long ws_rows;
@@ -807,6 +810,18 @@ __device__ __forceinline__ void tma_role(const Params &p, const Cta &c, const in
                 const int row0_i = __shfl_sync(0xffffffffu, row0, i);
                 const int src_i = __shfl_sync(0xffffffffu, src, i);
                 const int kv_i = __shfl_sync(0xffffffffu, kv, i);
+                if (p.l2_prefetch && w.mode == 0) {      // tiles that come from DRAM: ask L2 for the one four loads ahead
+                    constexpr int KVP_L2_PREFETCH = 4;
+                    const int j = min(i + KVP_L2_PREFETCH, 31);
+                    const int row0_j = __shfl_sync(0xffffffffu, row0, j);
+                    const int src_j = __shfl_sync(0xffffffffu, src, j);
+                    const int kv_j = __shfl_sync(0xffffffffu, kv, j);
+                    if (lane == 0 && i + KVP_L2_PREFETCH < cnt && src_j != 2) {
+                        const CUtensorMap *tm = src_j == 0 ? (kv_j ? tm_pool_v : tm_pool_k) : (kv_j ? tm_ws_v : tm_ws_k);
+                        asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(0), "r"(row0_j), "r"(w.plane) : "memory");
+                        asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(64), "r"(row0_j), "r"(w.plane) : "memory");
+                    }
+                }
                 if (lane == 0) {
                     const uint32_t g = ring_n + (uint32_t)(q0 + i);
                     const uint32_t stage = g % kStages, use = g / kStages;
@@ -1283,6 +1298,7 @@ cudaError_t kvp_launch_attn_sm100(const kvp_shape &sh, const kvp_attn2_args &a, 
     p.status = a.status;
     p.tail_direct = a.tail_direct;
     p.precise = a.precise;
+    p.l2_prefetch = a.l2_prefetch;
     p.k_new = (const uint4 *)a.k_new;
     p.v_new = (const uint4 *)a.v_new;
     p.ws_k = (uint4 *)a.ws_k;

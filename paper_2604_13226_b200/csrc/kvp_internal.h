@@ -219,6 +219,7 @@ struct kvp_attn2_args {
     // tm_knew / tm_vnew and the kernel copies those rows into the workspace rows itself
     int32_t tail_direct;
     int32_t precise;               // KVP_PRECISE_QK
+    int32_t l2_prefetch;           // the launch has at most two 256-row units per (request, kv head)
     const void *k_new, *v_new;
     char *ws_k, *ws_v;
     CUtensorMap tm_knew, tm_vnew;
