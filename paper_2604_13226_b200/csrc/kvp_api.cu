@@ -202,9 +202,11 @@ int find_slot(kvp_ctx *ctx, int32_t assembly_id)
 // rows of one request and kv head) are laid end to end, each weighted by the tensor-core work of its
 // key tiles, and the line is cut into equal shares, one per CTA; a cut closer than two tiles to a unit
 // boundary moves onto it.  A unit that ends up in several pieces gets partial slots and merge items.
-// Start-up and write-out of a piece (first Q tile, pipeline fill, epilogue) cost about as much as four
-// two-stream key tiles; the unit weights carry it so that CTAs with more pieces get fewer tiles.
-constexpr int kPieceCost = 8;
+// Start-up and write-out of a piece (first Q tile, pipeline fill, epilogue) cost about as much as two
+// two-stream key tiles (measured: 7,000 cycles per piece against 3,500-4,000 per tile pair, from the
+// per-CTA durations of a config-3 launch); the unit weights carry it so that CTAs with more pieces get
+// fewer tiles.  Counted in single-stream tiles.
+constexpr int kPieceCost = 4;
 
 struct schedule_t {
     std::vector<int32_t> cta_begin;
@@ -222,7 +224,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
 {
     const kvp_shape &sh = ctx->shape;
     const bool force_partial = (opts & KVP_PARTIAL) != 0, skip_tail = (opts & KVP_SKIP_QUERY_BLOCK) != 0;
-    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces, q_len, t_first; };
+    struct unit_t { int32_t b, hk, row_base, mode, n_all, first_piece, n_pieces, q_len, t_first, tile_begin, tail_row0; };
     std::vector<unit_t> units;
     const int max_rows = sh.group * q_len;
     int64_t total = 0;
@@ -244,6 +246,8 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 const int n_tail = (q_pos0 + last / sh.group) / KVP_TILE_KEYS + 1;
                 u.n_all = n_tail + n_prefix;
                 u.t_first = skip_tail ? n_tail : 0;
+                u.tile_begin = item.tile_begin;
+                u.tail_row0 = item.tail_row0;
                 u.first_piece = u.n_pieces = 0;
                 units.push_back(u);
                 total += (int64_t)(u.n_all - u.t_first) * (u.mode ? 1 : 2) + kPieceCost;
@@ -253,18 +257,31 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
     if (ctx->split_target_ctas > 0) G = std::min(ctx->split_target_ctas, kMaxCtas);
     const bool no_split = ctx->force_splits == 1;               // cuts only between units
 
-    // Cut positions (unit, tile), non-decreasing.  CTAs are filled one after the other up to a budget;
-    // every piece pays kPieceCost on top of its tiles, a piece is at least two tiles long (or the whole
-    // unit), and without splitting a unit goes to the CTA that holds its larger part.  The smallest
-    // budget that needs no more than G CTAs is found by bisection.
+    // Cut positions (unit, tile), non-decreasing.  A run of units is dealt out to g CTAs one after the other, each
+    // taking its even share of what is left (the work still to hand out divided by the CTAs still to fill, but
+    // not less than a minimum that keeps tiny launches on few CTAs); every piece pays kPieceCost on top of its
+    // tiles, a piece is at least two tiles long (or the whole unit), and without splitting a unit goes to the CTA
+    // that holds its larger part.  The last CTA of the run takes all that is left, so g CTAs always suffice.
     struct cut_t { int32_t u, t; };
     std::vector<cut_t> cuts;
-    auto fill = [&](size_t u_begin, size_t u_end, int64_t budget, std::vector<cut_t> *rec) -> int {
+    const int64_t min_budget = 8 + kPieceCost;
+    auto fill = [&](size_t u_begin, size_t u_end, int g, std::vector<cut_t> *rec) -> int {
+        std::vector<int64_t> after(u_end - u_begin + 1, 0);           // weight of the units behind unit u
+        for (size_t u = u_end; u > u_begin; --u) {
+            const unit_t &x = units[u - 1];
+            const int64_t wgt = x.n_all == x.t_first ? 0 : (int64_t)(x.n_all - x.t_first) * (x.mode ? 1 : 2) + kPieceCost;
+            after[u - 1 - u_begin] = after[u - u_begin] + wgt;
+        }
         int used = 0;
         size_t u = u_begin;
         while (u < u_end && units[u].n_all == units[u].t_first) ++u;      // units without a key tile get no piece
         int32_t t = u < u_end ? units[u].t_first : 0;
         while (u < u_end) {
+            const int64_t left_all = after[u + 1 - u_begin] + (int64_t)(units[u].n_all - t) * (units[u].mode ? 1 : 2) + kPieceCost;
+            const int ctas_left = std::max(1, g - used);
+            // every further CTA is likely to start inside a unit, i.e. to add a piece
+            const int64_t to_share = left_all + (int64_t)kPieceCost * (ctas_left - 1);
+            const int64_t budget = ctas_left == 1 ? left_all : std::max(min_budget, (to_share + ctas_left - 1) / ctas_left);
             ++used;
             if (rec) rec->push_back({(int32_t)u, t});
             int64_t cost = 0;
@@ -272,7 +289,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
                 const int w = units[u].mode ? 1 : 2;
                 const int32_t left = units[u].n_all - t;
                 const int64_t room = budget - cost - kPieceCost;
-                int32_t take = (int32_t)std::min<int64_t>(left, room > 0 ? (room + w - 1) / w : 0);
+                int32_t take = (int32_t)std::min<int64_t>(left, room > 0 ? room / w : 0);      // rounded down: the shares are re-dealt at every CTA
                 if (no_split) take = (t == units[u].t_first && (2 * take >= left || cost == 0)) ? left : 0;
                 if (left - take < 2) take = left;                 // do not leave a sliver behind
                 if (take < 2 && take < left) take = 0;
@@ -294,12 +311,8 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
         return used;
     };
     auto cut_range = [&](size_t u_begin, size_t u_end, int64_t weight, int g) {
-        int64_t lo_b = std::max<int64_t>(weight / g, 8 + kPieceCost), hi_b = weight + kPieceCost;
-        while (lo_b < hi_b) {
-            const int64_t mid = (lo_b + hi_b) / 2;
-            if (fill(u_begin, u_end, mid, nullptr) <= g) hi_b = mid; else lo_b = mid + 1;
-        }
-        fill(u_begin, u_end, lo_b, &cuts);
+        (void)weight;
+        fill(u_begin, u_end, g, &cuts);
     };
     // Each row block gets its own run of CTAs, in proportion to its work, and is cut on its own: row blocks of
     // equal work then get the same cuts, so the CTAs of units that share K/V walk the same tiles in step.  With
@@ -357,6 +370,7 @@ int32_t plan_schedule(kvp_ctx *ctx, const kvp_assembly_host &as, int layer, int 
             w.b = units[u].b; w.hk = units[u].hk; w.row_base = units[u].row_base;
             w.mode = units[u].mode | (units[u].q_len << 8);       // a request's own query length rides in the upper bits
             w.tile_lo = lo; w.n_tiles = hi - lo; w.slot0 = w.slot1 = -1;
+            w.tile_begin = units[u].tile_begin; w.tail_row0 = units[u].tail_row0; w.pad[0] = w.pad[1] = 0;
             rec.ws.push_back(w);
             rec.unit.push_back(u);
         }
@@ -1301,7 +1315,8 @@ int32_t kvp_export_schedule(kvp_ctx *ctx, int32_t assembly_id, int32_t q_len, in
     if ((cta_begin && cta_cap < sc.n_ctas + 1) || (works && work_cap < counts[1]) || (merges && merge_cap < counts[2]))
         return fail(ctx, KVP_ERR_CAPACITY, "export_schedule: output arrays too small");
     if (cta_begin) memcpy(cta_begin, sc.cta_begin.data(), 4 * sc.cta_begin.size());
-    if (works) memcpy(works, sc.works.data(), sizeof(kvp_work) * sc.works.size());
+    if (works)
+        for (size_t i = 0; i < sc.works.size(); ++i) memcpy(works + 8 * i, &sc.works[i], 32);     // the 8 documented ints of a piece
     if (merges) memcpy(merges, sc.merges.data(), sizeof(kvp_merge_item) * sc.merges.size());
     return KVP_OK;
 }

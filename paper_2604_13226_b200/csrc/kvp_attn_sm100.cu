@@ -293,15 +293,13 @@ struct Work {
 __device__ __forceinline__ Work load_work(const Params &p, int wi)
 {
     const int4 *w4 = reinterpret_cast<const int4 *>(p.works + wi);
-    const int4 a = __ldg(w4), c = __ldg(w4 + 1);
+    const int4 a = __ldg(w4), c = __ldg(w4 + 1), e = __ldg(w4 + 2);
     Work w;
     w.b = a.x; w.hk = a.y; w.row_base = a.z; w.mode = a.w & 0xff;
     w.q_len = (a.w >> 8) ? (a.w >> 8) : p.q_len;
     w.lo = c.x; w.n = c.y; w.slot0 = c.z; w.slot1 = c.w;
-    const int4 *i4 = reinterpret_cast<const int4 *>(p.plan.items + (p.layer * p.n_kv + w.hk) * p.plan.item_stride + w.b);
-    const int4 ia = __ldg(i4), ib = __ldg(i4 + 1);          // prefix_len, tile_begin, tile_end, seg_begin | seg_end, tail_row0, ..
-    w.tile_begin = ia.y;
-    w.tail_row0 = ib.y;
+    w.tile_begin = e.x;                                       // the plan item's entries, carried in the work record
+    w.tail_row0 = e.y;
     const int n_rows = p.group * w.q_len;
     const int last = min(n_rows - 1, w.row_base + (w.mode ? KVP_TILE_ROWS : 2 * KVP_TILE_ROWS) - 1);
     w.n_tail = (p.q_pos0 + last / p.group) / KVP_TILE_KEYS + 1;

@@ -64,7 +64,12 @@ struct kvp_work {
     int32_t mode;
     int32_t tile_lo, n_tiles;  // range in the unit's tile numbering
     int32_t slot0, slot1;      // stream 0 / stream 1 (mode 1 uses slot0 only)
+    // copied from the request's plan item, so that a CTA's first look-up is one memory round trip, not two
+    int32_t tile_begin;        // first prefix tile of the (request, plane) in the plan's tile array
+    int32_t tail_row0;         // workspace row where the request's query K/V rows are appended
+    int32_t pad[2];
 };
+static_assert(sizeof(kvp_work) == 48, "three 16-byte words");
 
 struct kvp_merge_item {        // 128 packed rows whose result is spread over n_slots partial slots
     int32_t b, hk;

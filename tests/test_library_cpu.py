@@ -229,8 +229,8 @@ def test_schedule_covers_every_tile_once(case):
         assert n >= 2 and row_base % 128 == 0 and row_base < n_rows
         named += list(range(s0, s0 + n))
     assert sorted(named) == list(range(n_slots))
-    # balance: no CTA carries more than its share plus a few tiles (a piece's fixed cost counts as 8)
-    cost = [sum(int(works[i][5]) * (1 if works[i][3] else 2) + 8 for i in range(cb[c], cb[c + 1])) for c in range(len(cb) - 1)]
+    # balance: no CTA carries more than its share plus a few tiles (a piece's fixed cost counts as 4)
+    cost = [sum(int(works[i][5]) * (1 if works[i][3] else 2) + 4 for i in range(cb[c], cb[c + 1])) for c in range(len(cb) - 1)]
     assert max(cost) <= sum(cost) / len(cost) + 16
 
 
