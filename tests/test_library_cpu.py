@@ -283,6 +283,31 @@ def test_schedule_gives_units_that_share_keys_the_same_cuts_on_neighbouring_ctas
     ctx.close()
 
 
+def test_row_blocks_with_different_causal_tiles_are_cut_at_the_same_prefix_tiles():
+    # 256 query tokens, g = 4: four 256-row units per (request, kv head) with 1, 1, 2, 2 causal tiles in front of
+    # the same 65 prefix tiles.  Counted from the first prefix tile the cuts of all row blocks coincide, and the j-th
+    # CTAs of the row blocks sit next to each other: CTAs that stream the same K/V stay on the same tiles.
+    ctx, aid, plen, shape = _schedule_case(32, 8, [2048] * 4, [[(i, 0) for i in range(4)]] * 2, 256)
+    cb, works, merges, n_slots = ctx.export_schedule(aid, 256)
+    n_ctas = len(cb) - 1
+    starts = {}
+    for c in range(n_ctas):
+        for i in range(cb[c], cb[c + 1]):
+            b, hk, row_base, mode, lo, n = (int(x) for x in works[i][:6])
+            last = min(4 * 256, row_base + 256) - 1
+            n_tail = (last // 4) // 128 + 1
+            starts.setdefault(row_base, []).append((b, hk, 0 if lo == 0 else lo - n_tail, c))
+    assert sorted(starts) == [0, 256, 512, 768]
+    ref = [(b, hk, p) for b, hk, p, c in starts[0]]
+    assert any(p > 0 for _, _, p in ref)                       # units are split
+    for rb, lst in starts.items():
+        assert [(b, hk, p) for b, hk, p, c in lst] == ref       # same cuts in prefix coordinates
+    for j in range(len(ref)):                                   # and the CTAs that share a cut are neighbours
+        ctas = [starts[rb][j][3] for rb in sorted(starts)]
+        assert max(ctas) - min(ctas) <= 2 * len(starts)
+    ctx.close()
+
+
 def test_packets_registered_from_host_memory_plan_like_any_other():
     # host-only context: nothing is copied, but rows are reserved in the same order and the plan is the same;
     # only packets that came from host memory can be evicted
