@@ -10,9 +10,14 @@ prints ONE JSON line.  ``value`` = query tokens/s of the whole job (batch * q_le
 full layer stack per step), inputs resident in HBM.  ``e2e`` = the same with the step's Q/K_new/V_new
 coming from pinned host buffers and the outputs read back, copies inside the timed region.
 ``roofline`` is for the dominant kernel (the tcgen05 attention kernel), its duration measured live
-with CUDA events on the launching stream.  ``extra_points`` add the memory-bound short-query shape, the
-gather kernel in materialise mode and a decode step (one token per request).  ``cpu_baseline`` is the fp64 oracle on the host cores on a
-bounded sample.  ``--impl reference`` times that oracle as the reference arm.
+with CUDA events on the launching stream; the fraction is given against the measured burst and sustained
+bf16 GEMM peaks and the nominal one, with the rule that picks the headline.  ``extra_points`` add the
+memory-bound short-query shape, the gather kernel in materialise mode, a decode step (one token per
+request), one layer of config 4, config 2, a pruned-packet layer and host-resident packets, each with the
+clock record of its own timed region.  ``cpu_baseline`` is the fp64 oracle on the host cores on a bounded
+sample.  ``--impl reference`` times that same sample as the reference arm.  ``--shard prefix`` is the second
+multi-GPU mode: the packets of one long-context batch split over the ranks, one all-gather of partial
+results per layer.
 
 Workloads (seeded, synthetic, shaped like the paper's Llama-3.1-8B / Qwen2.5-7B RAG requests):
 config3 (default; Llama-3.1-8B 32-layer stack, 10 x 1024-token packets, 128 query tokens, batch 4),
