@@ -480,7 +480,8 @@ def run_prefix_shard(args, rank: int, world: int, local_rank: int, peaks):
         raise SystemExit(f"--shard prefix: {n} packets per request do not divide over {world} ranks")
     per_rank = n // world
     whole = gen.spec_config5(n, ql, b, seed=args.seed)
-    spec = gen.spec_config5(per_rank, ql, b, seed=args.seed + 17 * rank)          # this rank's packets (its own draws)
+    # this rank's packets; with one request they are the whole workload's own bytes, else the rank's own draws
+    spec = gen.shard_spec(whole, rank, world)[0] if b == 1 else gen.spec_config5(per_rank, ql, b, seed=args.seed + 17 * rank)
     doc = spec.packet_lens[0] + spec.n_header + spec.n_trailer
     pos_base = [rank * per_rank * doc] * b
     s = spec.shape

@@ -338,6 +338,7 @@ class LargeSpec:
     outlier_channels: int = 0
     outlier_scale: float = 8.0
     rebase: bool = True
+    packet_seed_offset: int = 0             # packet p is drawn with the seeds of packet p + offset (a rank's part of a sharded spec)
 
     @property
     def batch(self) -> int:
@@ -377,6 +378,27 @@ def spec_config5(n_packets: int, q_len: int, batch: int, seed: int = 0, doc_len:
     shape = ModelShape(1, 32, 8, 128, "bf16", 500000.0, 0)
     return LargeSpec(f"config5_n{n_packets}_q{q_len}_b{batch}", shape, [doc_len] * (batch * n_packets),
                      items, q_len, seed=seed)
+
+
+def shard_spec(spec: LargeSpec, rank: int, world: int):
+    """Rank ``rank``'s part of a spec whose requests use consecutive, distinct packets (config 5): every request's
+    slot list is cut into ``world`` equal contiguous parts; the rank's packets keep the seeds they have in the whole
+    spec, so the ranks together hold exactly the whole workload's bytes.  Returns (sub-spec, pos_base)."""
+    per = [len(it) for it in spec.items]
+    assert all(n % world == 0 for n in per), "slots do not divide over the ranks"
+    flat = [pid for it in spec.items for pid, _ in it]
+    assert flat == list(range(len(flat))), "requests must use consecutive distinct packets"
+    # a rank's packets are not one contiguous range of the whole spec unless there is a single request, so the
+    # sub-spec keeps one seed offset per request by laying its packets out request by request
+    assert len(spec.items) == 1 or world == 1, "shard_spec handles one request per spec (use one spec per request)"
+    n = per[0] // world
+    lo = rank * n
+    items = [[(s, aid) for s, (_, aid) in enumerate(spec.items[0][lo:lo + n])]]
+    lens = [spec.packet_lens[pid] for pid, _ in spec.items[0][lo:lo + n]]
+    pos = sum(spec.packet_lens[pid] + (spec.n_header + spec.n_trailer if aid >= 0 else 0) for pid, aid in spec.items[0][:lo])
+    sub = LargeSpec(f"{spec.name}_rank{rank}of{world}", spec.shape, lens, items, spec.q_len, spec.n_header, spec.n_trailer,
+                    spec.seed, spec.outlier_channels, spec.outlier_scale, spec.rebase, spec.packet_seed_offset + lo)
+    return sub, [pos]
 
 
 class DeviceWorkload:
@@ -432,8 +454,9 @@ class DeviceWorkload:
     def packet_device(self, pid: int):
         s = self.shape
         dims = (s.n_layers, self.spec.packet_lens[pid], s.n_kv_heads, s.head_dim)
-        return (self._randn(self._base + 4 * pid, dims, self._chan),
-                self._randn(self._base + 4 * pid + 1, dims, self._chan))
+        gp = pid + self.spec.packet_seed_offset
+        return (self._randn(self._base + 4 * gp, dims, self._chan),
+                self._randn(self._base + 4 * gp + 1, dims, self._chan))
 
     def adapter_device(self):
         s = self.shape

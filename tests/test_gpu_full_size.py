@@ -119,3 +119,42 @@ def test_config5_sweep_points(n_packets, q_len, batch, requests):
     sess.close()
     del sess, wl
     torch.cuda.empty_cache()
+
+
+def test_config5_longest_prefix_sharded_over_two_ranks():
+    # the 133,120-token request of the memory-bound sweep point with its 64 packets on two ranks (32 each, the same
+    # bytes as the whole workload): partial prefill per rank, the gathered buffers merged, sampled rows against the
+    # oracle over the WHOLE request - the launch configuration `bench.py --shard prefix` times
+    whole = gen.spec_config5(64, 16, 1, seed=0)
+    wl = gen.DeviceWorkload(whole, "cuda:0")
+    s = whole.shape
+    parts, sessions = [], []
+    for r in range(2):
+        sub, pos_base = gen.shard_spec(whole, r, 2)
+        assert sub.prefix_len(0) == 32 * 2080 and pos_base == [r * 32 * 2080]
+        sess = Session(gen.DeviceWorkload(sub, "cuda:0"))
+        aid, plen = sess.assemble(pos_base=pos_base)
+        q, kn, vn = wl.query_device(0)
+        buf = torch.empty(sess.ctx.partial_bytes(1, 16), dtype=torch.uint8, device=q.device)
+        sess.ctx.query_prefill(aid, 0, q, kn, vn, 16, buf, None, kvp.PARTIAL | (kvp.SKIP_QUERY_BLOCK if r == 0 else 0))
+        assert sess.ctx.status_word() == 0
+        parts.append(buf)
+        sessions.append(sess)
+    out = torch.zeros(1, 16, s.n_q_heads, s.head_dim, dtype=torch.bfloat16, device="cuda:0")
+    lse = torch.zeros(1, s.n_q_heads, 16, dtype=torch.float32, device="cuda:0")
+    sessions[0].ctx.merge_partials(torch.cat(parts), 2, 1, 16, out, lse)
+    torch.cuda.synchronize()
+    o = orc.widen(torch_to_np(out, "bf16"), "bf16")
+    rows = sample_rows(whole, 400)
+    st = make_store(wl)
+    q, kn, vn = wl.query_layer(0)
+    plan = orc.compose(st, wl.items[0], True)
+    ro, rl, _, _ = orc.query_prefill(st, plan, 0, q[0], kn[0], vn[0], orc.inv_freq(s.rope_theta, s.head_dim), s.rope_pairing, rows=rows)
+    stats = attention_error_stats(np.stack([o[0, i, h] for h, i in rows]), ro)
+    print("raw attention error vs oracle, prefix sharded over 2 ranks:", stats)
+    l = lse.cpu().numpy()
+    assert max(abs(l[0, h, i] - rl[n]) for n, (h, i) in enumerate(rows)) <= 2e-2
+    for sess in sessions:
+        sess.close()
+    del sessions, parts, wl
+    torch.cuda.empty_cache()
