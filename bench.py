@@ -17,7 +17,7 @@ request), one layer of config 4, config 2, a pruned-packet layer and host-reside
 clock record of its own timed region.  ``cpu_baseline`` is the fp64 oracle on the host cores on a bounded
 sample.  ``--impl reference`` times that same sample as the reference arm.  ``--shard prefix`` is the second
 multi-GPU mode: the packets of one long-context batch split over the ranks, one all-gather of partial
-results per layer.
+results per layer.  ``--shard heads`` is the third: the kv heads of one batch split over the ranks, no exchange.
 
 Workloads (seeded, synthetic, shaped like the paper's Llama-3.1-8B / Qwen2.5-7B RAG requests):
 config3 (default; Llama-3.1-8B 32-layer stack, 10 x 1024-token packets, 128 query tokens, batch 4),
@@ -130,9 +130,18 @@ def max_over_ranks(values, world: int, device=None):
     return [float(x) for x in t]
 
 
-def job_tokens_per_s(spec, world: int, ms_step: float) -> float:
-    """Whole-job rate: every rank pushes batch * q_len query tokens through the stack per step."""
-    return spec.batch * spec.q_len * world / (ms_step * 1e-3)
+def head_spec(workload: str, seed: int, rank: int, world: int):
+    """`--shard heads`: rank `rank` holds kv heads [rank Hkv / world, (rank + 1) Hkv / world) of every packet of the
+    SAME batch, and the query heads that read them (strong scaling; attention is independent per kv head, so there is
+    no exchange inside the path - the ranks' outputs are the head slices of the output)."""
+    from paper_2604_13226_b200 import inputs as gen
+    return gen.shard_heads_spec(make_spec(workload, seed), rank, world)
+
+
+def job_tokens_per_s(spec, world: int, ms_step: float, shard: str = "requests") -> float:
+    """Whole-job rate: with requests sharded every rank pushes its own batch * q_len query tokens through the stack
+    per step; with heads sharded all ranks work on the same batch * q_len tokens."""
+    return spec.batch * spec.q_len * (world if shard == "requests" else 1) / (ms_step * 1e-3)
 
 
 class ClockSampler:
@@ -269,16 +278,20 @@ def prefill_flags(spec) -> int:
     return kvp.PRECISE_QK if getattr(spec, "outlier_channels", 0) else 0
 
 
-def workload_config(spec, materialize: bool, bytes_per_layer: float):
+def workload_config(spec, materialize: bool, bytes_per_layer: float, shard: str = "requests", world: int = 1):
     """The `config` object of the JSON line: the workload, named the same way by both arms."""
     s = spec.shape
+    sharding = "requests sharded across ranks, no collective"
+    if shard == "heads":
+        sharding = ("kv heads sharded across ranks (%d of %d kv heads and their %d query heads per GPU, the same batch on "
+                    "every rank), no collective" % (s.n_kv_heads, s.n_kv_heads * world, s.n_q_heads))
     return {"workload": spec.name, "layers": s.n_layers, "q_heads": s.n_q_heads, "kv_heads": s.n_kv_heads,
             "head_dim": s.head_dim, "batch_per_gpu": spec.batch, "q_len": spec.q_len,
             "prefix_tokens": [spec.prefix_len(b) for b in range(spec.batch)], "rope_theta": s.rope_theta,
             "mode": "materialised cache" if materialize else "fused in place (adapters staged)",
             "qk": "precise (KVP_PRECISE_QK)" if prefill_flags(spec) else "plain",
             "l2": "inputs larger than L2: every layer reads %.0f MB of distinct K/V" % (bytes_per_layer / 1e6),
-            "sharding": "requests sharded across ranks, no collective"}
+            "sharding": sharding}
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -605,9 +618,10 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the extra roofline points and the CPU baseline")
     ap.add_argument("--materialize", action="store_true", help="materialise the composed prefix instead of reading in place")
-    ap.add_argument("--shard", default="requests", choices=["requests", "prefix"],
+    ap.add_argument("--shard", default="requests", choices=["requests", "prefix", "heads"],
                     help="requests: every rank its own batch (weak scaling, the default); prefix: the packets of one "
-                         "long-context batch (config5:<packets>:<q_len>:<batch>) split over the ranks (strong scaling)")
+                         "long-context batch (config5:<packets>:<q_len>:<batch>) split over the ranks (strong scaling); "
+                         "heads: the kv heads of one batch split over the ranks, no exchange (strong scaling)")
     ap.add_argument("--sweep", action="store_true",
                     help="time the attention kernel over the config-5 grid (packets x q_len x batch) and print one JSON line per point")
     args = ap.parse_args()
@@ -686,7 +700,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    spec = rank_spec(args.workload, args.seed, rank)               # weak scaling: every rank its own batch
+    by_heads = args.shard == "heads"
+    # weak scaling: every rank its own batch; or strong scaling over the kv heads of one batch
+    spec = head_spec(args.workload, args.seed, rank, world) if by_heads else rank_spec(args.workload, args.seed, rank)
     s = spec.shape
     wl = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
     sess = Session(wl, materialize=args.materialize, device=local_rank)
@@ -798,16 +814,16 @@ def main():
     torch.cuda.empty_cache()
 
     if rank == 0:
-        tokens = spec.batch * Lq * world
+        tokens = spec.batch * Lq * (1 if by_heads else world)
         ms_step = ms_total / args.steps
-        value = job_tokens_per_s(spec, world, ms_step)
+        value = job_tokens_per_s(spec, world, ms_step, args.shard)
         flops, bytes_ = algorithmic_work(spec)
         a_ms = statistics.mean(attn_ms) if attn_ms else None
         tensor_bound = s.group * Lq >= 247
         traffic = None
         tpath = os.path.join(ROOT, "profiles", "roofline_traffic.json")
         if os.path.exists(tpath):
-            traffic = json.load(open(tpath)).get(spec.name)
+            traffic = None if (by_heads and world > 1) else json.load(open(tpath)).get(spec.name)   # counters: all heads on one GPU
         if a_ms:
             if tensor_bound:
                 ach = flops / a_ms / 1e9
@@ -829,10 +845,11 @@ def main():
         line = {
             "metric": "composed_cache_prefill_query_tokens_per_s", "value": value, "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32",
+            "higher_is_better": True, "scaling": "strong" if by_heads else "weak", "vs_baseline": None,
+            "dtype": "bf16" if s.dtype == "bf16" else "f32",
             "data": "synthetic",
-            "config": workload_config(spec, args.materialize, bytes_),
-            "prefix_tokens_per_s": sum(spec.prefix_len(b) for b in range(spec.batch)) * world / (ms_step * 1e-3),
+            "config": workload_config(spec, args.materialize, bytes_, args.shard, world),
+            "prefix_tokens_per_s": sum(spec.prefix_len(b) for b in range(spec.batch)) * (1 if by_heads else world) / (ms_step * 1e-3),
             "e2e": {"value": tokens / (ms_e2e / args.steps * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e / args.steps,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches_per_step * args.steps, "launch": launch, "roofline": roof, "clocks": clocks,

@@ -226,6 +226,28 @@ def shard_workload(wl: Workload, rank: int, world: int):
     return sub, pos_base
 
 
+def shard_heads(wl: Workload, rank: int, world: int) -> Workload:
+    """Rank ``rank``'s part of a workload sharded by kv head over ``world`` ranks: kv heads
+    [rank * Hkv / world, (rank + 1) * Hkv / world) of every packet, adapter and query tensor, with the query heads
+    that read them.  Plain slicing: attention is independent per kv head, so the ranks' outputs put side by side
+    along the head axis are the whole workload's output."""
+    s = wl.shape
+    assert s.n_kv_heads % world == 0, "kv heads do not divide over the ranks"
+    n_kv = s.n_kv_heads // world
+    h0, h1 = rank * n_kv, (rank + 1) * n_kv
+    g = s.group
+    shape = ModelShape(s.n_layers, n_kv * g, n_kv, s.head_dim, s.dtype, s.rope_theta, s.rope_pairing)
+    cut = lambda a: np.ascontiguousarray(a[..., h0:h1, :])
+    packets = []
+    for pk in wl.packets:
+        kept = None if pk.kept is None else [list(layer[h0:h1]) for layer in pk.kept]
+        packets.append(Packet(cut(pk.k), cut(pk.v), pk.cache_pos0, kept))
+    adapters = [Adapter(cut(a.hk), cut(a.hv), cut(a.tk), cut(a.tv), a.header_pos0, a.trailer_pos0) for a in wl.adapters]
+    q = np.ascontiguousarray(wl.q[..., h0 * g:h1 * g, :])
+    return Workload(shape, packets, adapters, [list(it) for it in wl.items], q, cut(wl.k_new), cut(wl.v_new), wl.rebase,
+                    f"{wl.name}_heads{rank}of{world}", wl.seed, dict(wl.notes))
+
+
 # --------------------------------------------------------------------------------------
 # small, numpy-drawn workloads
 # --------------------------------------------------------------------------------------
@@ -399,6 +421,18 @@ def shard_spec(spec: LargeSpec, rank: int, world: int):
     sub = LargeSpec(f"{spec.name}_rank{rank}of{world}", spec.shape, lens, items, spec.q_len, spec.n_header, spec.n_trailer,
                     spec.seed, spec.outlier_channels, spec.outlier_scale, spec.rebase, spec.packet_seed_offset + lo)
     return sub, [pos]
+
+
+def shard_heads_spec(spec: LargeSpec, rank: int, world: int) -> LargeSpec:
+    """Rank ``rank``'s part of a spec sharded by kv head: the same requests and packet lengths with Hkv / world kv
+    heads (and their query heads), drawn with the rank's own seed - every rank holds different heads' values."""
+    s = spec.shape
+    assert s.n_kv_heads % world == 0, "kv heads do not divide over the ranks"
+    n_kv = s.n_kv_heads // world
+    shape = ModelShape(s.n_layers, n_kv * s.group, n_kv, s.head_dim, s.dtype, s.rope_theta, s.rope_pairing)
+    return LargeSpec(spec.name, shape, list(spec.packet_lens), [list(it) for it in spec.items], spec.q_len, spec.n_header,
+                     spec.n_trailer, spec.seed + 17 * rank, spec.outlier_channels, spec.outlier_scale, spec.rebase,
+                     spec.packet_seed_offset)
 
 
 class DeviceWorkload:

@@ -123,3 +123,72 @@ def test_two_gloo_ranks_plan_the_parts_of_prefix_sharded_requests(tmp_path):
         assert d["ok"] and d["tiles"] and d["total"] == d["whole"]
         # 3 requests x 2 kv heads x 1 row tile of 128 packed rows, 64 fp32 columns + (m, l) per row
         assert d["partial_bytes"] == 3 * 2 * 1 * 128 * (64 * 4 + 8)
+
+
+# Kv-head sharding: every rank plans the SAME requests for its own heads; the head ranges tile [0, Hkv), the ranks'
+# slices put side by side are the whole tensors, the composition (which rows, which offsets) does not depend on the
+# heads, and the whole-job rate counts the batch once.
+HEAD_WORKER = r'''
+import json, os, sys
+sys.path.insert(0, os.environ["KVP_ROOT"]); sys.path.insert(0, os.path.join(os.environ["KVP_ROOT"], "tests"))
+import numpy as np
+import torch.distributed as dist
+from oracle import reference as orc
+import bench
+from paper_2604_13226_b200 import binding as kvp, inputs as gen
+from helpers import make_store
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", rank=rank, world_size=world)
+shape = gen.ModelShape(2, 12, 4, 64, "f32", 10000.0, 0)
+items = [[(0, 0), (1, 0), (2, -1)], [(2, 0), (0, 0)]]
+wl = gen.make_workload(shape, [40, 130, 7], items, q_len=5, n_header=3, n_trailer=5, seed=11, packet_pos0=[0, 11, 2])
+sub = gen.shard_heads(wl, rank, world)
+s = sub.shape
+ctx = kvp.Context(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.dtype, rope_theta=s.rope_theta, max_packets=4,
+                  max_adapters=1, max_batch=2, max_slots=8, max_prefix_tokens=512, max_query_tokens=5, max_ws_rows=1024, device=-1)
+for p in sub.packets:
+    ctx.register_packet(None, None, p.n_tokens, p.cache_pos0)
+a = sub.adapters[0]
+ctx.register_adapter(None, None, a.n_header, a.header_pos0, None, None, a.n_trailer, a.trailer_pos0)
+aid, plen = ctx.assemble(sub.items, kvp.REBASE)
+st = make_store(wl)                                              # the whole workload's store: the plan must not depend on the heads
+ok = plen == [wl.prefix_len(b) for b in range(wl.batch)]
+for b in range(wl.batch):
+    whole = orc.compose(st, wl.items[b])
+    src, dl, segs = ctx.export_plan(aid, b)
+    ok = ok and np.array_equal(dl, whole.delta) and len(segs) == len(whole.segments)
+    ok = ok and all(int(g[1]) == int(m[1]) and int(g[2]) == int(m[2]) and int(g[3]) == int(m[3]) for g, m in zip(segs, whole.segments))
+gathered = [None] * world
+dist.all_gather_object(gathered, (sub.q, sub.k_new, sub.packets[1].k, sub.adapters[0].tv))
+whole_again = [np.concatenate([g[i] for g in gathered], axis=-2) for i in range(4)]
+tiles = all(np.array_equal(x, y) for x, y in zip(whole_again, (wl.q, wl.k_new, wl.packets[1].k, wl.adapters[0].tv)))
+spec = bench.head_spec("config3", 0, rank, world)
+ms = bench.max_over_ranks([4.0 + rank], world)
+print(json.dumps({"rank": rank, "ok": bool(ok), "tiles": bool(tiles), "heads": [s.n_q_heads, s.n_kv_heads],
+                  "spec_heads": [spec.shape.n_q_heads, spec.shape.n_kv_heads], "spec_seed": spec.seed, "items": spec.items,
+                  "value": bench.job_tokens_per_s(spec, world, ms[0], "heads")}))
+dist.destroy_process_group()
+'''
+
+
+def test_two_gloo_ranks_shard_kv_heads_of_the_same_requests(tmp_path):
+    script = tmp_path / "head_worker.py"
+    script.write_text(HEAD_WORKER)
+    port = 33500 + os.getpid() % 2000
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port),
+                   KVP_ROOT=ROOT, CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=240)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(json.loads(out.strip().splitlines()[-1]))
+    outs.sort(key=lambda d: d["rank"])
+    a, b = outs
+    assert a["ok"] and b["ok"] and a["tiles"] and b["tiles"]
+    assert a["heads"] == b["heads"] == [6, 2]                       # 12 / 4 heads over two ranks, g = 3 kept
+    assert a["spec_heads"] == b["spec_heads"] == [16, 4]            # config 3: 32 / 8 heads over two ranks
+    assert a["items"] == b["items"] and a["spec_seed"] != b["spec_seed"]      # the same requests, each rank its heads' values
+    assert abs(a["value"] - 4 * 128 / 5.0e-3) < 1e-6 and a["value"] == b["value"]   # the batch counted once, slowest rank
