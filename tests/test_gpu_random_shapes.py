@@ -76,3 +76,57 @@ def test_random_shapes_chunked_continuation(seed):
     d = (both.float() - whole.float()).abs()
     assert float(d.max()) <= 3e-2 and float(d.mean()) <= 2e-3
     sess.close()
+
+
+def random_large_workload(seed):
+    rng = np.random.default_rng(5000 + seed)
+    n_kv = int(rng.choice([1, 2, 4, 8]))
+    group = int(rng.choice([1, 4, 7, 8]))
+    shape = gen.ModelShape(1, n_kv * group, n_kv, 128, "bf16", 500000.0, int(rng.integers(0, 2)))
+    n_packets = int(rng.integers(1, 9))
+    lens = [int(rng.choice([1, 64, 129, 700, 1024, 2048, 3000])) for _ in range(n_packets)]
+    batch = int(rng.integers(1, 5))
+    items = [[(int(rng.integers(0, n_packets)), int(rng.choice([0, 0, -1]))) for _ in range(int(rng.integers(0, 7)))]
+             for _ in range(batch)]
+    if all(len(it) == 0 for it in items):
+        items[0] = [(0, 0)]
+    q_len = int(rng.choice([5, 128, 300, 512, 777, 1024]))
+    keep = None
+    if rng.integers(0, 4) == 0:                                 # a quarter of the cases with pruned packets
+        keep = [float(rng.choice([0.1, 0.5, 0.9])) if rng.integers(0, 2) else None for _ in range(n_packets)]
+    wl = gen.make_workload(shape, lens, items, q_len=q_len, seed=seed, keep_rate=keep)
+    cuts = sorted(set([0, q_len] + [int(x) for x in rng.integers(1, q_len, size=2)]))
+    return wl, int(rng.choice([0, 0, 5, 60, 148])), keep is not None, cuts
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_large_shapes_long_queries_pruned_packets_and_three_chunk_continuation(seed):
+    # Longer queries (many query tiles per kv head, several causal tiles), longer and pruned documents, up to 8 kv
+    # heads: the tcgen05 kernel against the CUDA-core kernel on every row (the oracle would take minutes here; the
+    # CUDA-core kernel is checked against it on the small cases above), then the same query in three calls.
+    wl, ctas, pruned, cuts = random_large_workload(seed)
+    sess = Session(wl)
+    if ctas:
+        sess.ctx.tune(kvp.TUNE_SPLIT_TARGET_CTAS, ctas)
+    sess.assemble()
+    q, kn, vn = sess.query_tensors(0)
+    out, lse = sess.prefill(0, qkv=(q, kn, vn))
+    assert sess.ctx.status_word() == 0 and sess.ctx.last_launch()["kind"] == 1
+    ref, ref_lse = sess.prefill(0, kvp.FORCE_SIMPLE, qkv=(q, kn, vn))
+    d = (out.float() - ref.float()).abs()
+    assert float(d.max()) <= 3e-2 and float(d.mean()) <= 2e-3, (seed, float(d.max()), float(d.mean()))
+    assert float((lse - ref_lse).abs().max()) <= 2e-2
+    if not pruned:
+        sess.assemble()
+        outs = []
+        for i in range(len(cuts) - 1):
+            a, b = cuts[i], cuts[i + 1]
+            qq, kk, vv = (t[:, a:b].contiguous() for t in (q, kn, vn))
+            o = torch.empty_like(qq)
+            sess.ctx.query_prefill(sess.assembly_id, 0, qq, kk, vv, b - a, o, None, kvp.CONTINUE if i else 0)
+            outs.append(o)
+        torch.cuda.synchronize()
+        assert sess.ctx.status_word() == 0
+        d = (torch.cat(outs, dim=1).float() - ref.float()).abs()
+        assert float(d.max()) <= 3e-2 and float(d.mean()) <= 2e-3, (seed, cuts, float(d.max()), float(d.mean()))
+    sess.close()
