@@ -192,3 +192,29 @@ def test_two_gloo_ranks_shard_kv_heads_of_the_same_requests(tmp_path):
     assert a["spec_heads"] == b["spec_heads"] == [16, 4]            # config 3: 32 / 8 heads over two ranks
     assert a["items"] == b["items"] and a["spec_seed"] != b["spec_seed"]      # the same requests, each rank its heads' values
     assert abs(a["value"] - 4 * 128 / 5.0e-3) < 1e-6 and a["value"] == b["value"]   # the batch counted once, slowest rank
+
+
+def test_oracle_over_head_slices_equals_slices_of_the_oracle_over_all_heads():
+    # What kv-head sharding rests on, checked on the oracle alone: the definition's result for query head h depends on
+    # kv head h // g only, so the oracle run on rank r's slice of a workload (inputs.shard_heads) gives, bit for bit,
+    # rank r's slice of the oracle's result for the whole workload - plain and with a pruned packet.
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from paper_2604_13226_b200 import inputs as gen
+    from helpers import oracle_outputs
+    shape = gen.ModelShape(2, 12, 4, 64, "f32", 10000.0, 1)
+    items = [[(0, 0), (1, 0), (2, -1)], [(2, 0), (0, 0)]]
+    for keep in (None, [0.5, None, 0.8]):
+        wl = gen.make_workload(shape, [40, 130, 7], items, q_len=5, n_header=3, n_trailer=5, seed=12, packet_pos0=[0, 11, 2],
+                               keep_rate=keep)
+        whole = oracle_outputs(wl, layer=1)
+        for world in (2, 4):
+            g, per = shape.group, shape.n_q_heads // world
+            for r in range(world):
+                part = oracle_outputs(gen.shard_heads(wl, r, world), layer=1)
+                for b in range(wl.batch):
+                    wo = whole[b][0].reshape(wl.q_len, shape.n_q_heads, shape.head_dim)[:, r * per:(r + 1) * per]
+                    wlse = whole[b][1].reshape(wl.q_len, shape.n_q_heads)[:, r * per:(r + 1) * per]
+                    assert np.array_equal(part[b][0].reshape(wl.q_len, per, shape.head_dim), wo)
+                    assert np.array_equal(part[b][1].reshape(wl.q_len, per), wlse)
