@@ -246,6 +246,12 @@ def oracle_sample(spec, wl, n_tokens: int = ORACLE_TOKENS):
     for pid, n in enumerate(spec.packet_lens):
         st.register_packet(n, 0, (lambda layer, pid=pid: cached[pid]))
     st.register_adapter(ad.n_header, 0, ad.n_trailer, 0, (lambda layer: (ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0])))
+    from paper_2604_13226_b200 import inputs as gen
+    pids = sorted(cached)
+    digests = {"algorithm": "blake2b-64 over the raw bytes, layer 0",
+               "q": gen.digest64(q), "k_new": gen.digest64(kn), "v_new": gen.digest64(vn),
+               "packets_k": gen.digest64(*[cached[p][0] for p in pids]), "packets_v": gen.digest64(*[cached[p][1] for p in pids]),
+               "adapter": gen.digest64(ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0]), "packets": len(pids)}
     toks = list(range(spec.q_len))
     if 0 < n_tokens < spec.q_len:
         toks = sorted({int(round(i * (spec.q_len - 1) / (n_tokens - 1))) for i in range(n_tokens)}) if n_tokens > 1 else [spec.q_len - 1]
@@ -269,7 +275,7 @@ def oracle_sample(spec, wl, n_tokens: int = ORACLE_TOKENS):
             "sample": f"layer 0 of all {spec.batch} requests: compose + re-base + widening of the prefix ({t_fixed:.2f} s) and "
                       f"attention rows of {len(toks)} of {spec.q_len} query tokens x {s.n_q_heads} heads ({t_att:.2f} s); "
                       f"attention scaled to {spec.q_len} tokens, the sum to {s.n_layers} layers",
-            "seconds": t_fixed + t_att}
+            "seconds": t_fixed + t_att, "input_digests": digests}
 
 
 def prefill_flags(spec) -> int:

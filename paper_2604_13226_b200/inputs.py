@@ -226,6 +226,16 @@ def shard_workload(wl: Workload, rank: int, world: int):
     return sub, pos_base
 
 
+def digest64(*arrays) -> str:
+    """64-bit BLAKE2b digest (hex) of the raw bytes of the given arrays, in order: what a report carries so that two
+    runs (or the two sides of one run) can tell whether they worked on the same input bytes."""
+    import hashlib
+    h = hashlib.blake2b(digest_size=8)
+    for a in arrays:
+        h.update(np.ascontiguousarray(a).view(np.uint8).reshape(-1).data)
+    return h.hexdigest()
+
+
 def shard_heads(wl: Workload, rank: int, world: int) -> Workload:
     """Rank ``rank``'s part of a workload sharded by kv head over ``world`` ranks: kv heads
     [rank * Hkv / world, (rank + 1) * Hkv / world) of every packet, adapter and query tensor, with the query heads

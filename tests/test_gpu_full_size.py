@@ -158,3 +158,21 @@ def test_config5_longest_prefix_sharded_over_two_ranks():
         sess.close()
     del sessions, parts, wl
     torch.cuda.empty_cache()
+
+
+def test_device_workload_redraws_the_same_bytes_and_a_second_instance_too():
+    # The large workloads are never stored: every tensor is re-drawn from its seed when it is needed - by the session
+    # that registers it, by the oracle that checks it, by the CPU baseline.  The digests a bench report carries are
+    # only worth something if a re-draw gives the same bytes: same object twice, a second object, device against host.
+    spec = gen.spec_config3(seed=5, n_layers=2, batch=2, pool=6, per_item=3, doc_len=300, q_len=16)
+    a, b = gen.DeviceWorkload(spec, "cuda:0"), gen.DeviceWorkload(spec, "cuda:0")
+    for pid in (0, 5):
+        k0, v0 = a.packet_layer(pid, 1)
+        k1, v1 = a.packet_layer(pid, 1)
+        k2, v2 = b.packet_layer(pid, 1)
+        kd, vd = a.packet_device(pid)
+        assert gen.digest64(k0, v0) == gen.digest64(k1, v1) == gen.digest64(k2, v2)
+        assert gen.digest64(k0) == gen.digest64(torch_to_np(kd[1], "bf16")) and gen.digest64(v0) == gen.digest64(torch_to_np(vd[1], "bf16"))
+    assert gen.digest64(*a.query_layer(1)) == gen.digest64(*b.query_layer(1)) != gen.digest64(*a.query_layer(0))
+    other = gen.DeviceWorkload(gen.spec_config3(seed=6, n_layers=2, batch=2, pool=6, per_item=3, doc_len=300, q_len=16), "cuda:0")
+    assert gen.digest64(*other.packet_layer(0, 1)) != gen.digest64(*a.packet_layer(0, 1))
