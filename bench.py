@@ -15,7 +15,7 @@ bf16 GEMM peaks and the nominal one, with the rule that picks the headline.  ``e
 memory-bound short-query shape, the gather kernel in materialise mode, a decode step (one token per
 request), one layer of config 4, config 2, a pruned-packet layer and host-resident packets, each with the
 clock record of its own timed region.  ``cpu_baseline`` is the fp64 oracle on the host cores on a bounded
-sample.  ``--impl reference`` times that same sample as the reference arm.  ``--shard prefix`` is the second
+sample (three layers, about 10 s).  ``--impl reference`` times a smaller sample of the same kind once per step.  ``--shard prefix`` is the second
 multi-GPU mode: the packets of one long-context batch split over the ranks, one all-gather of partial
 results per layer.  ``--shard heads`` is the third: the kv heads of one batch split over the ranks, no exchange.
 
@@ -222,60 +222,75 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------------
 
 ORACLE_TOKENS = 32          # query tokens per request the oracle is timed on (evenly spaced over the chunk)
+BASELINE_TOKENS = 64        # the same for the `cpu_baseline` object, which also takes three layers (about 10 s of CPU work)
 
 
-def oracle_sample(spec, wl, n_tokens: int = ORACLE_TOKENS):
-    """Time the fp64 oracle, as it stands, on layer 0 of every request: composition + re-basing of the whole
+def oracle_sample(spec, wl, n_tokens: int = ORACLE_TOKENS, layers=(0,)):
+    """Time the fp64 oracle, as it stands, on the given layers of every request: composition + re-basing of the whole
     prefix and the widening / concatenation of its inputs (a fixed cost per request and layer), then attention
     for every head of `n_tokens` query tokens spread evenly over the chunk (0 = all).  Only the attention time is
-    scaled to the full chunk (work per row is the same to within q_len / prefix).  Returns the job-level rate it
-    implies: query tokens/s through the full stack = batch*q_len / (L * sum_b t_b).  `cpu_baseline` and the
-    reference arm both call this with the default sample."""
+    scaled to the full chunk (work per row is the same to within q_len / prefix), and the mean over the sampled
+    layers to the stack.  Returns the job-level rate it implies: query tokens/s through the full stack =
+    batch*q_len / (L * mean_l sum_b t_b).  The reference arm times the default sample once per step; `cpu_baseline`
+    times a larger one (first, middle and last layer, twice the tokens)."""
     from oracle import reference as orc
+    from paper_2604_13226_b200 import inputs as gen
     s = spec.shape
     ad = wl.adapter_host()
     f = orc.inv_freq(s.rope_theta, s.head_dim)
-    q, kn, vn = wl.query_layer(0)
-    # pull the bytes to the host before timing (the oracle's inputs are host arrays)
-    cached = {}
-    for it in spec.items:
-        for pid, _ in it:
-            if pid not in cached:
-                cached[pid] = wl.packet_layer(pid, 0)
-    st = orc.Store(s.dtype)
-    for pid, n in enumerate(spec.packet_lens):
-        st.register_packet(n, 0, (lambda layer, pid=pid: cached[pid]))
-    st.register_adapter(ad.n_header, 0, ad.n_trailer, 0, (lambda layer: (ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0])))
-    from paper_2604_13226_b200 import inputs as gen
-    pids = sorted(cached)
-    digests = {"algorithm": "blake2b-64 over the raw bytes, layer 0",
-               "q": gen.digest64(q), "k_new": gen.digest64(kn), "v_new": gen.digest64(vn),
-               "packets_k": gen.digest64(*[cached[p][0] for p in pids]), "packets_v": gen.digest64(*[cached[p][1] for p in pids]),
-               "adapter": gen.digest64(ad.hk[0], ad.hv[0], ad.tk[0], ad.tv[0]), "packets": len(pids)}
     toks = list(range(spec.q_len))
     if 0 < n_tokens < spec.q_len:
         toks = sorted({int(round(i * (spec.q_len - 1) / (n_tokens - 1))) for i in range(n_tokens)}) if n_tokens > 1 else [spec.q_len - 1]
     rows = [(h, i) for i in toks for h in range(s.n_q_heads)]
+    layers = sorted({min(max(int(l), 0), s.n_layers - 1) for l in layers})
     t_total = t_fixed = t_att = 0.0
-    for b in range(spec.batch):
-        t0 = time.perf_counter()
-        plan = orc.compose(st, spec.items[b], spec.rebase)
-        Kp, Vp, _ = orc.composed_kv(st, plan, 0, f, s.rope_pairing)
-        Q = orc.widen(q[b], s.dtype)
-        K = np.concatenate([Kp, orc.widen(kn[b], s.dtype)])
-        V = np.concatenate([Vp, orc.widen(vn[b], s.dtype)])
-        t1 = time.perf_counter()
-        orc.attention_rows(K, V, Q, plan.prefix_len, 1.0 / np.sqrt(s.head_dim), rows)
-        t2 = time.perf_counter()
-        t_fixed += t1 - t0
-        t_att += t2 - t1
-        t_total += (t1 - t0) + (t2 - t1) / len(rows) * (spec.q_len * s.n_q_heads)
-    tokens_per_s = spec.batch * spec.q_len / (s.n_layers * t_total)
+    digests = None
+    for layer in layers:
+        q, kn, vn = wl.query_layer(layer)
+        # pull the bytes to the host before timing (the oracle's inputs are host arrays)
+        cached = {}
+        for it in spec.items:
+            for pid, _ in it:
+                if pid not in cached:
+                    cached[pid] = wl.packet_layer(pid, layer)
+        st = orc.Store(s.dtype)
+        for pid, n in enumerate(spec.packet_lens):
+            st.register_packet(n, 0, (lambda l_, pid=pid: cached[pid]))
+        st.register_adapter(ad.n_header, 0, ad.n_trailer, 0,
+                            (lambda l_, layer=layer: (ad.hk[layer], ad.hv[layer], ad.tk[layer], ad.tv[layer])))
+        if digests is None:
+            pids = sorted(cached)
+            digests = {"algorithm": "blake2b-64 over the raw bytes, layer %d" % layer,
+                       "q": gen.digest64(q), "k_new": gen.digest64(kn), "v_new": gen.digest64(vn),
+                       "packets_k": gen.digest64(*[cached[p][0] for p in pids]),
+                       "packets_v": gen.digest64(*[cached[p][1] for p in pids]),
+                       "adapter": gen.digest64(ad.hk[layer], ad.hv[layer], ad.tk[layer], ad.tv[layer]), "packets": len(pids)}
+        for b in range(spec.batch):
+            t0 = time.perf_counter()
+            plan = orc.compose(st, spec.items[b], spec.rebase)
+            Kp, Vp, _ = orc.composed_kv(st, plan, layer, f, s.rope_pairing)
+            Q = orc.widen(q[b], s.dtype)
+            K = np.concatenate([Kp, orc.widen(kn[b], s.dtype)])
+            V = np.concatenate([Vp, orc.widen(vn[b], s.dtype)])
+            t1 = time.perf_counter()
+            orc.attention_rows(K, V, Q, plan.prefix_len, 1.0 / np.sqrt(s.head_dim), rows)
+            t2 = time.perf_counter()
+            t_fixed += t1 - t0
+            t_att += t2 - t1
+            t_total += (t1 - t0) + (t2 - t1) / len(rows) * (spec.q_len * s.n_q_heads)
+    tokens_per_s = spec.batch * spec.q_len / (s.n_layers * t_total / len(layers))
     return {"value": tokens_per_s, "unit": "tokens/s", "cores": orc.threads(), "kind": "oracle",
-            "sample": f"layer 0 of all {spec.batch} requests: compose + re-base + widening of the prefix ({t_fixed:.2f} s) and "
-                      f"attention rows of {len(toks)} of {spec.q_len} query tokens x {s.n_q_heads} heads ({t_att:.2f} s); "
-                      f"attention scaled to {spec.q_len} tokens, the sum to {s.n_layers} layers",
+            "sample": f"layer{'s' if len(layers) > 1 else ''} {', '.join(str(l) for l in layers)} of all {spec.batch} requests: compose + "
+                      f"re-base + widening of the prefix ({t_fixed:.2f} s) and attention rows of {len(toks)} of {spec.q_len} query "
+                      f"tokens x {s.n_q_heads} heads ({t_att:.2f} s); attention scaled to {spec.q_len} tokens, the mean over the "
+                      f"sampled layers to {s.n_layers} layers",
             "seconds": t_fixed + t_att, "input_digests": digests}
+
+
+def baseline_sample(spec, wl):
+    """The `cpu_baseline` object: the oracle on the first, middle and last layer, BASELINE_TOKENS query tokens each."""
+    L = spec.shape.n_layers
+    return oracle_sample(spec, wl, n_tokens=BASELINE_TOKENS, layers=(0, L // 2, L - 1))
 
 
 def prefill_flags(spec) -> int:
@@ -669,7 +684,7 @@ def main():
         for _ in range(args.warmup):
             oracle_sample(spec, wl, n_tokens=1)
         t0 = time.perf_counter()
-        vals = [oracle_sample(spec, wl) for _ in range(max(1, args.steps))]      # the sample cpu_baseline times
+        vals = [oracle_sample(spec, wl) for _ in range(max(1, args.steps))]      # one bounded sample per step
         dt = time.perf_counter() - t0
         v = statistics.median(x["value"] for x in vals)
         cb = dict(vals[-1])
@@ -876,7 +891,7 @@ def main():
                 extras["error"] = repr(ex)
             line["extra_points"] = extras
             wl2 = gen.DeviceWorkload(spec, f"cuda:{local_rank}")
-            line["cpu_baseline"] = oracle_sample(spec, wl2)
+            line["cpu_baseline"] = baseline_sample(spec, wl2)
         sampler.stop()
         print(json.dumps(line))
     if world > 1:
